@@ -1,0 +1,166 @@
+/*
+ * qesgd.h -- C ABI of the B200 (sm_100a) QESGD hot path.
+ *
+ * Quantized Epoch-SGD (Zhao, Gao, Li, arXiv 1901.03040) compresses the epoch
+ * delta z = u - w_t of a parameter vector against the server's anchor w_t
+ * with a uniform stochastic quantiser and averages the quantised deltas on the
+ * server.  This library is that data path on one GPU:
+ *
+ *   worker side   qesgd_encode[_batch]         delta, per-bucket scale, stochastic
+ *                                              rounding to s levels, sign+level packing
+ *   server side   qesgd_decode_average_apply   decode K streams, average, add to w_t
+ *                 qesgd_decode                 decode one stream to fp32
+ *   local epoch   qesgd_lr_sgd_step / qesgd_lr_local_epoch[_batch]
+ *                                              logistic-regression minibatch SGD
+ *
+ * Conventions
+ *   - Every data pointer is a DEVICE pointer owned by the caller and valid on
+ *     the context's device, unless marked "host".  The library never frees or
+ *     reallocates caller memory.  Vectors (local, anchor, param, out, X, u) need
+ *     4-byte alignment; 32-byte alignment of the base pointers and of the
+ *     per-worker strides selects the fast 256-bit load path.  Code and scale
+ *     buffers must be 16-byte aligned and their per-worker strides multiples of
+ *     16 bytes.
+ *   - Calls enqueue work on the context's stream and return without waiting;
+ *     only qesgd_status and qesgd_destroy synchronise.
+ *   - Return value: QESGD_OK or a negative error code.  Nothing is enqueued
+ *     when an error is returned.  No call aborts or throws.
+ *   - Data problems (a non-finite value in a bucket) never fail a call: the
+ *     bucket is encoded as scale 0 / codes 0 and QESGD_STATUS_NONFINITE is set
+ *     in the context's status word, read with qesgd_status.
+ *   - Element counts d are 64-bit; d == 0 is a valid no-op.
+ *
+ * Stream format (shared by encode and decode)
+ *   bucket j covers elements [j*bucket, (j+1)*bucket); the last bucket is padded
+ *   with zeros; nb = ceil(d/bucket).  A worker's stream is nb*bucket codes of
+ *   `bits` bits (bits in {2,4,8}; top bit = sign, low bits-1 bits = level in
+ *   [0, s]); element e occupies bits [(e mod (32/bits))*bits, +bits) of the
+ *   little-endian 32-bit word e/(32/bits).  Padding codes are 0.  Its scales are
+ *   nb floats; a decoded value is +-level * fl32(scale/s).
+ */
+#ifndef QESGD_H
+#define QESGD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define QESGD_OK 0
+#define QESGD_EINVAL (-1) /* NULL / misaligned pointer, unsupported bits, bucket, s, K, mode */
+#define QESGD_ECUDA (-2)  /* CUDA runtime or launch error; see qesgd_last_cuda_error      */
+#define QESGD_ENOMEM (-3) /* host or device allocation failed (qesgd_create only)          */
+
+#define QESGD_SCALE_NORM 0u  /* scale = L2 norm of the bucket's delta              */
+#define QESGD_SCALE_MAX 1u   /* scale = largest magnitude of the bucket's delta    */
+#define QESGD_SCALE_FIXED 2u /* scale = s*delta with the grid spacing delta given  */
+
+#define QESGD_STATUS_NONFINITE 1u /* a bucket held NaN/Inf or its norm overflowed fp32 */
+
+#define QESGD_MAX_WORKERS 64u
+#define QESGD_MIN_BUCKET 64u
+#define QESGD_MAX_BUCKET 8192u
+#define QESGD_MAX_LR_BATCH 1024u
+
+typedef struct qesgd_ctx qesgd_ctx;
+
+/* Create a context bound to `device` and to `cuda_stream` (a cudaStream_t passed
+ * as void*; NULL = the legacy default stream).  Allocates a few KB of device
+ * memory (status word, logistic-regression workspace) that qesgd_destroy frees.
+ * This is the only call that allocates. */
+int qesgd_create(qesgd_ctx **out, int device, void *cuda_stream);
+int qesgd_destroy(qesgd_ctx *ctx);
+/* Rebind the context to another stream of the same device. */
+int qesgd_set_stream(qesgd_ctx *ctx, void *cuda_stream);
+
+/* ceil(d / bucket); 0 for an invalid bucket. */
+uint64_t qesgd_num_buckets(uint64_t d, uint32_t bucket);
+/* Bytes of one worker's code stream: nb * bucket * bits / 8 (a multiple of 16). */
+uint64_t qesgd_code_bytes(uint64_t d, uint32_t bucket, uint32_t bits);
+
+/*
+ * Worker side (paper Sec. 2.2: compress z = u - w_t; Sec. 3: bucket remark;
+ * Eq. 4: stochastic rounding; Eq. 3: b-bit grid).
+ *
+ *   z_i   = fl32(local_i - anchor_i), or local_i when anchor == NULL
+ *   scale = fl32(sqrt(sum z_i^2))  (NORM; fp64 sum over the balanced binary tree on
+ *           index order)  |  max |z_i|  (MAX)  |  fl32(s*fixed_delta)  (FIXED)
+ *   r_i   = min(fl32(|z_i| * fl32(s/scale)), s);  level_i = floor(r_i) + [u_i < frac(r_i)]
+ *   u_i   = (h_i + 1/2) / 2^16 with h_i the 16-bit draw of element i from
+ *           Philox4x32-10, counter (i>>3 low, i>>3 high, worker, epoch), key = seed,
+ *           32-bit word (i>>1)&3, half (i&1)
+ *   code  = sign<<(bits-1) | level, sign = (z_i < 0 and level > 0)
+ * A bucket with scale < 2^-100 or non-finite content is written as scale 0, codes 0.
+ *
+ * local, anchor: float[d] (anchor may be NULL).  codes_out: qesgd_code_bytes()
+ * bytes.  scales_out: float[nb].  All nb*bucket codes and nb scales are written.
+ * s in [1, 2^(bits-1)-1]; bucket a power of two in [64, 8192]; fixed_delta is
+ * read only for QESGD_SCALE_FIXED and must then be finite and > 0.
+ */
+int qesgd_encode(qesgd_ctx *ctx, const float *local, const float *anchor, uint64_t d,
+                 uint32_t bucket, uint32_t s, uint32_t bits, uint32_t scale_mode,
+                 float fixed_delta, uint64_t seed, uint32_t worker, uint32_t epoch,
+                 uint32_t *codes_out, float *scales_out);
+
+/* K workers in one launch (K simulated workers of Algorithm 3 on one device):
+ * worker k reads local + k*local_stride (elements) against the shared anchor,
+ * draws with worker id worker0 + k, writes codes_out + k*code_stride (BYTES) and
+ * scales_out + k*scale_stride (elements).  1 <= K <= 64. */
+int qesgd_encode_batch(qesgd_ctx *ctx, const float *local, uint64_t local_stride,
+                       const float *anchor, uint64_t d, uint32_t K, uint32_t bucket, uint32_t s,
+                       uint32_t bits, uint32_t scale_mode, float fixed_delta, uint64_t seed,
+                       uint32_t worker0, uint32_t epoch, uint32_t *codes_out,
+                       uint64_t code_stride, float *scales_out, uint64_t scale_stride);
+
+/*
+ * Server side (last line of the server task of Algorithm 3, same average as the
+ * last line of Algorithms 1 and 2):
+ *   param_i <- param_i + (1/K) * sum_k (+-level_{k,i} * fl32(scale_{k,bucket(i)} / s))
+ * param: float[d], updated in place, read once and written once.  Stream k starts
+ * at codes + k*code_stride (BYTES) and scales + k*scale_stride (elements).
+ * fp32 accumulation; result within 1e-6 * max(|param_i|, max_k scale) of the
+ * exactly rounded value.  1 <= K <= 64.
+ */
+int qesgd_decode_average_apply(qesgd_ctx *ctx, float *param, uint64_t d, uint32_t K,
+                               const uint32_t *codes, uint64_t code_stride, const float *scales,
+                               uint64_t scale_stride, uint32_t bucket, uint32_t s, uint32_t bits);
+
+/* Decoding alone (the grid points delta*k of Eq. 3): out_i = +-level_i *
+ * fl32(scale/s), i < d, bit-exact.  out: float[d]. */
+int qesgd_decode(qesgd_ctx *ctx, const uint32_t *codes, const float *scales, uint64_t d,
+                 uint32_t bucket, uint32_t s, uint32_t bits, float *out);
+
+/*
+ * Local epoch on logistic regression (Sec. 1: f_i(w) = log(1 + exp(-y_i x_i^T w));
+ * Eq. 2: u <- u - (lr/m) * sum_j grad f_j(u); worker task of Algorithm 3).
+ * One step on the m rows of Xb (row-major float[m][d]) with labels yb (float[m],
+ * +-1): u (float[d]) is updated in place.  fp32 arithmetic, fp32 accumulation.
+ * 1 <= m <= QESGD_MAX_LR_BATCH.
+ */
+int qesgd_lr_sgd_step(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32_t m, uint64_t d,
+                      float lr, float *u);
+/* Rows [0, n_local) of X in consecutive minibatches of `batch` rows, in row
+ * order; a last partial batch uses its own size in Eq. 2. */
+int qesgd_lr_local_epoch(qesgd_ctx *ctx, const float *X, const float *y, uint64_t n_local,
+                         uint64_t d, uint32_t batch, float lr, float *u);
+/* K workers side by side: worker k owns rows [k*n_local, (k+1)*n_local) of X and
+ * y and updates u + k*u_stride (elements).  Step t of every worker runs in the
+ * same launches. */
+int qesgd_lr_local_epoch_batch(qesgd_ctx *ctx, const float *X, const float *y, uint64_t n_local,
+                               uint64_t d, uint32_t K, uint32_t batch, float lr, float *u,
+                               uint64_t u_stride);
+
+/* Waits for the stream, copies the status word to *flags_out (host) and clears it. */
+int qesgd_status(qesgd_ctx *ctx, uint32_t *flags_out);
+/* Number of kernels this context has launched since creation. */
+uint64_t qesgd_launch_count(const qesgd_ctx *ctx);
+/* Last cudaError_t seen by this context (0 if none). */
+int qesgd_last_cuda_error(const qesgd_ctx *ctx);
+/* Static text for a return code. */
+const char *qesgd_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QESGD_H */

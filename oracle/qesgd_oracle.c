@@ -181,7 +181,17 @@ int qesgd_ref_encode(const float *local, const float *anchor, uint64_t n, uint64
             uint64_t idx = lo + e;
             float v = 0.0f;
             if (idx < n) v = anchor ? local[idx] - anchor[idx] : local[idx];
-            if (!isfinite(v)) finite = 0;
+            if (scale_mode == QREF_SCALE_FIXED) {
+                /* Nothing couples the elements of a bucket here.  +-Inf lies beyond
+                 * the range and clips like any large value (first and last branch of
+                 * Eq. 4); NaN has no place on the grid: flagged, encoded as 0. */
+                if (isnan(v)) {
+                    if (status) *status |= QREF_STATUS_NONFINITE;
+                    v = 0.0f;
+                }
+            } else if (!isfinite(v)) {
+                finite = 0;
+            }
             z[e] = v;
         }
         float scale;

@@ -1,0 +1,307 @@
+// C ABI of libqesgd.so: context management, argument validation, dispatch.
+// Contracts are stated in include/qesgd.h.
+#include <new>
+
+#include "qesgd_internal.h"
+
+namespace {
+
+inline bool aligned(const void *p, uintptr_t a) { return ((uintptr_t)p % a) == 0; }
+
+inline int log2_exact(uint32_t v)
+{
+    int l = 0;
+    while ((1u << l) < v) ++l;
+    return l;
+}
+
+inline bool valid_bucket(uint32_t b)
+{
+    return b >= QESGD_MIN_BUCKET && b <= QESGD_MAX_BUCKET && (b & (b - 1u)) == 0u;
+}
+
+inline bool valid_codec(uint32_t bucket, uint32_t s, uint32_t bits)
+{
+    if (!(bits == 2 || bits == 4 || bits == 8)) return false;
+    if (!valid_bucket(bucket)) return false;
+    return s >= 1u && s <= (1u << (bits - 1)) - 1u;
+}
+
+// Binds the context's device for the duration of a call and restores the caller's.
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int device)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == device) || cudaSetDevice(device) == cudaSuccess;
+        if (prev == device) prev = -1;
+    }
+    ~DeviceGuard()
+    {
+        if (ok && prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+int cuda_fail(qesgd_ctx *ctx, int err)
+{
+    ctx->last_cuda_error = err;
+    return QESGD_ECUDA;
+}
+
+}  // namespace
+
+extern "C" {
+
+int qesgd_create(qesgd_ctx **out, int device, void *cuda_stream)
+{
+    if (!out) return QESGD_EINVAL;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess) return QESGD_ECUDA;
+    if (device < 0 || device >= count) return QESGD_EINVAL;
+    qesgd_ctx *ctx = new (std::nothrow) qesgd_ctx();
+    if (!ctx) return QESGD_ENOMEM;
+    ctx->device = device;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    ctx->launches = 0;
+    ctx->last_cuda_error = 0;
+    ctx->d_status = nullptr;
+    ctx->d_lr_work = nullptr;
+    ctx->lr_work_floats = QESGD_LR_WORK_FLOATS;
+    DeviceGuard guard(device);
+    if (!guard.ok) { delete ctx; return QESGD_ECUDA; }
+    cudaError_t e = cudaMalloc((void **)&ctx->d_status, 256);
+    if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->d_lr_work, ctx->lr_work_floats * sizeof(float));
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
+    if (e == cudaSuccess)
+        e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
+    if (e != cudaSuccess) {
+        cudaFree(ctx->d_status);
+        cudaFree(ctx->d_lr_work);
+        delete ctx;
+        return e == cudaErrorMemoryAllocation ? QESGD_ENOMEM : QESGD_ECUDA;
+    }
+    *out = ctx;
+    return QESGD_OK;
+}
+
+int qesgd_destroy(qesgd_ctx *ctx)
+{
+    if (!ctx) return QESGD_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (guard.ok) {
+        cudaStreamSynchronize(ctx->stream);
+        cudaFree(ctx->d_status);
+        cudaFree(ctx->d_lr_work);
+    }
+    delete ctx;
+    return guard.ok ? QESGD_OK : QESGD_ECUDA;
+}
+
+int qesgd_set_stream(qesgd_ctx *ctx, void *cuda_stream)
+{
+    if (!ctx) return QESGD_EINVAL;
+    ctx->stream = (cudaStream_t)cuda_stream;
+    return QESGD_OK;
+}
+
+uint64_t qesgd_num_buckets(uint64_t d, uint32_t bucket)
+{
+    if (!valid_bucket(bucket)) return 0;
+    return (d + bucket - 1) / bucket;
+}
+
+uint64_t qesgd_code_bytes(uint64_t d, uint32_t bucket, uint32_t bits)
+{
+    if (!valid_bucket(bucket) || !(bits == 2 || bits == 4 || bits == 8)) return 0;
+    return qesgd_num_buckets(d, bucket) * (bucket / 8u) * bits;
+}
+
+int qesgd_encode_batch(qesgd_ctx *ctx, const float *local, uint64_t local_stride,
+                       const float *anchor, uint64_t d, uint32_t K, uint32_t bucket, uint32_t s,
+                       uint32_t bits, uint32_t scale_mode, float fixed_delta, uint64_t seed,
+                       uint32_t worker0, uint32_t epoch, uint32_t *codes_out,
+                       uint64_t code_stride, float *scales_out, uint64_t scale_stride)
+{
+    if (!ctx) return QESGD_EINVAL;
+    if (!valid_codec(bucket, s, bits) || scale_mode > QESGD_SCALE_FIXED) return QESGD_EINVAL;
+    if (K < 1 || K > QESGD_MAX_WORKERS) return QESGD_EINVAL;
+    if (scale_mode == QESGD_SCALE_FIXED && !(fixed_delta > 0.0f && fixed_delta <= 3.402823466e38f))
+        return QESGD_EINVAL;
+    if (d == 0) return QESGD_OK;
+    if (!local || !codes_out || !scales_out) return QESGD_EINVAL;
+    if (!aligned(local, 4) || !aligned(anchor, 4)) return QESGD_EINVAL;
+    if (!aligned(codes_out, 16) || !aligned(scales_out, 16)) return QESGD_EINVAL;
+    const uint64_t nb = qesgd_num_buckets(d, bucket);
+    const uint64_t cbytes = qesgd_code_bytes(d, bucket, bits);
+    if (K > 1) {
+        if (local_stride < d || code_stride < cbytes || scale_stride < nb) return QESGD_EINVAL;
+        if (code_stride % 16 != 0 || (scale_stride * 4) % 16 != 0) return QESGD_EINVAL;
+    }
+    EncodeArgs a;
+    a.local = local;
+    a.local_stride = K > 1 ? local_stride : 0;
+    a.anchor = anchor;
+    a.d = d;
+    a.padded = nb * bucket;
+    a.log2_bucket = (uint32_t)log2_exact(bucket);
+    a.s = s;
+    a.fixed_scale = scale_mode == QESGD_SCALE_FIXED ? (float)s * fixed_delta : 0.0f;
+    a.key0 = (uint32_t)seed;
+    a.key1 = (uint32_t)(seed >> 32);
+    a.worker0 = worker0;
+    a.epoch = epoch;
+    a.codes = codes_out;
+    a.code_stride = K > 1 ? code_stride : 0;
+    a.scales = scales_out;
+    a.scale_stride = K > 1 ? scale_stride : 0;
+    a.status = ctx->d_status;
+    const bool vec = aligned(local, 32) && aligned(anchor, 32) && (a.local_stride % 8 == 0);
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
+    const int e = qesgd_launch_encode(a, K, bits, scale_mode, vec, ctx->stream);
+    if (e != 0) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return QESGD_OK;
+}
+
+int qesgd_encode(qesgd_ctx *ctx, const float *local, const float *anchor, uint64_t d,
+                 uint32_t bucket, uint32_t s, uint32_t bits, uint32_t scale_mode,
+                 float fixed_delta, uint64_t seed, uint32_t worker, uint32_t epoch,
+                 uint32_t *codes_out, float *scales_out)
+{
+    return qesgd_encode_batch(ctx, local, 0, anchor, d, 1, bucket, s, bits, scale_mode,
+                              fixed_delta, seed, worker, epoch, codes_out, 0, scales_out, 0);
+}
+
+int qesgd_decode_average_apply(qesgd_ctx *ctx, float *param, uint64_t d, uint32_t K,
+                               const uint32_t *codes, uint64_t code_stride, const float *scales,
+                               uint64_t scale_stride, uint32_t bucket, uint32_t s, uint32_t bits)
+{
+    if (!ctx) return QESGD_EINVAL;
+    if (!valid_codec(bucket, s, bits)) return QESGD_EINVAL;
+    if (K < 1 || K > QESGD_MAX_WORKERS) return QESGD_EINVAL;
+    if (d == 0) return QESGD_OK;
+    if (!param || !codes || !scales) return QESGD_EINVAL;
+    if (!aligned(param, 4) || !aligned(codes, 16) || !aligned(scales, 16)) return QESGD_EINVAL;
+    const uint64_t nb = qesgd_num_buckets(d, bucket);
+    if (K > 1) {
+        if (code_stride < qesgd_code_bytes(d, bucket, bits) || scale_stride < nb) return QESGD_EINVAL;
+        if (code_stride % 16 != 0 || (scale_stride * 4) % 16 != 0) return QESGD_EINVAL;
+    }
+    DecodeArgs a;
+    a.param = param;
+    a.d = d;
+    a.nb = nb;
+    a.K = K;
+    a.log2_bucket = (uint32_t)log2_exact(bucket);
+    a.s = s;
+    a.codes = codes;
+    a.code_stride = K > 1 ? code_stride : 0;
+    a.scales = scales;
+    a.scale_stride = K > 1 ? scale_stride : 0;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
+    const int e = qesgd_launch_decode_average_apply(a, bits, aligned(param, 32), ctx->stream);
+    if (e != 0) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return QESGD_OK;
+}
+
+int qesgd_decode(qesgd_ctx *ctx, const uint32_t *codes, const float *scales, uint64_t d,
+                 uint32_t bucket, uint32_t s, uint32_t bits, float *out)
+{
+    if (!ctx) return QESGD_EINVAL;
+    if (!valid_codec(bucket, s, bits)) return QESGD_EINVAL;
+    if (d == 0) return QESGD_OK;
+    if (!out || !codes || !scales) return QESGD_EINVAL;
+    if (!aligned(out, 4) || !aligned(codes, 16) || !aligned(scales, 16)) return QESGD_EINVAL;
+    DecodeArgs a;
+    a.param = out;
+    a.d = d;
+    a.nb = qesgd_num_buckets(d, bucket);
+    a.K = 1;
+    a.log2_bucket = (uint32_t)log2_exact(bucket);
+    a.s = s;
+    a.codes = codes;
+    a.code_stride = 0;
+    a.scales = scales;
+    a.scale_stride = 0;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
+    const int e = qesgd_launch_decode(a, bits, aligned(out, 32), ctx->stream);
+    if (e != 0) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return QESGD_OK;
+}
+
+int qesgd_lr_local_epoch_batch(qesgd_ctx *ctx, const float *X, const float *y, uint64_t n_local,
+                               uint64_t d, uint32_t K, uint32_t batch, float lr, float *u,
+                               uint64_t u_stride)
+{
+    if (!ctx) return QESGD_EINVAL;
+    if (K < 1 || K > QESGD_MAX_WORKERS) return QESGD_EINVAL;
+    if (batch < 1 || batch > QESGD_MAX_LR_BATCH) return QESGD_EINVAL;
+    if (n_local == 0 || d == 0) return QESGD_OK;
+    if (!X || !y || !u) return QESGD_EINVAL;
+    if (!aligned(X, 4) || !aligned(y, 4) || !aligned(u, 4)) return QESGD_EINVAL;
+    if (K > 1 && u_stride < d) return QESGD_EINVAL;
+    const uint32_t m_max = (uint32_t)(n_local < batch ? n_local : batch);
+    if ((uint64_t)K * m_max > ctx->lr_work_floats) return QESGD_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
+    for (uint64_t r = 0; r < n_local; r += batch) {
+        const uint32_t m = (uint32_t)(n_local - r < batch ? n_local - r : batch);
+        int launched = 0;
+        const int e = qesgd_launch_lr_step(X + r * d, n_local * d, y + r, n_local, m, d, K, lr, u,
+                                           K > 1 ? u_stride : 0, ctx->d_lr_work,
+                                           ctx->lr_work_floats, ctx->stream, &launched);
+        ctx->launches += (uint64_t)launched;
+        if (e != 0) return cuda_fail(ctx, e);
+    }
+    return QESGD_OK;
+}
+
+int qesgd_lr_local_epoch(qesgd_ctx *ctx, const float *X, const float *y, uint64_t n_local,
+                         uint64_t d, uint32_t batch, float lr, float *u)
+{
+    return qesgd_lr_local_epoch_batch(ctx, X, y, n_local, d, 1, batch, lr, u, 0);
+}
+
+int qesgd_lr_sgd_step(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32_t m, uint64_t d,
+                      float lr, float *u)
+{
+    if (m < 1 || m > QESGD_MAX_LR_BATCH) return QESGD_EINVAL;
+    return qesgd_lr_local_epoch_batch(ctx, Xb, yb, m, d, 1, m, lr, u, 0);
+}
+
+int qesgd_status(qesgd_ctx *ctx, uint32_t *flags_out)
+{
+    if (!ctx || !flags_out) return QESGD_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
+    cudaError_t e = cudaMemcpyAsync(flags_out, ctx->d_status, sizeof(uint32_t),
+                                    cudaMemcpyDeviceToHost, ctx->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof(uint32_t), ctx->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
+    return QESGD_OK;
+}
+
+uint64_t qesgd_launch_count(const qesgd_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+int qesgd_last_cuda_error(const qesgd_ctx *ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+const char *qesgd_strerror(int code)
+{
+    switch (code) {
+        case QESGD_OK: return "ok";
+        case QESGD_EINVAL: return "invalid argument";
+        case QESGD_ECUDA: return "CUDA error (see qesgd_last_cuda_error)";
+        case QESGD_ENOMEM: return "out of memory";
+        default: return "unknown error";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,65 @@
+// Internal declarations shared by the translation units of libqesgd.so.
+// Nothing here is part of the public ABI (that is include/qesgd.h).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "qesgd.h"
+
+struct qesgd_ctx {
+    int device;
+    cudaStream_t stream;
+    uint32_t *d_status;     // device status word (bit set by kernels)
+    float *d_lr_work;       // logistic-regression partial margins
+    uint64_t lr_work_floats;
+    uint64_t launches;
+    int last_cuda_error;
+    int sm_count;
+};
+
+// Workspace for partial margins: K * P * m floats must fit.
+static const uint64_t QESGD_LR_WORK_FLOATS = 1ull << 20;
+
+struct EncodeArgs {
+    const float *local;
+    uint64_t local_stride;  // elements between workers
+    const float *anchor;    // may be null
+    uint64_t d;             // elements per worker
+    uint64_t padded;        // nb * bucket
+    uint32_t log2_bucket;
+    uint32_t s;
+    float fixed_scale;      // fl32(s * delta), FIXED mode only
+    uint32_t key0, key1;    // seed low / high
+    uint32_t worker0, epoch;
+    uint32_t *codes;
+    uint64_t code_stride;   // bytes between workers
+    float *scales;
+    uint64_t scale_stride;  // elements between workers
+    uint32_t *status;
+};
+
+struct DecodeArgs {
+    float *param;           // decode-average-apply: in/out; decode: out
+    uint64_t d;
+    uint64_t nb;
+    uint32_t K;
+    uint32_t log2_bucket;
+    uint32_t s;
+    const uint32_t *codes;
+    uint64_t code_stride;   // bytes
+    const float *scales;
+    uint64_t scale_stride;  // elements
+};
+
+// Launchers (defined in qesgd_codec.cu / qesgd_lr.cu).  Return a cudaError_t as int.
+int qesgd_launch_encode(const EncodeArgs &a, uint32_t K, uint32_t bits, uint32_t scale_mode,
+                        bool vec, cudaStream_t stream);
+int qesgd_launch_decode(const DecodeArgs &a, uint32_t bits, bool vec, cudaStream_t stream);
+int qesgd_launch_decode_average_apply(const DecodeArgs &a, uint32_t bits, bool vec,
+                                      cudaStream_t stream);
+// One minibatch step for K workers; returns the number of kernels launched in *launched.
+int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float *yb,
+                         uint64_t y_worker_stride, uint32_t m, uint64_t d, uint32_t K, float lr,
+                         float *u, uint64_t u_stride, float *work, uint64_t work_floats,
+                         cudaStream_t stream, int *launched);

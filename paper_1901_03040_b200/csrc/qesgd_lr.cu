@@ -1,0 +1,178 @@
+// Logistic-regression minibatch SGD step for sm_100a (paper Sec. 1: f_i(w) =
+// log(1 + exp(-y_i x_i^T w)); Eq. 2: u <- u - (lr/m) sum_j grad f_j(u)).
+//
+// Two streaming passes over the minibatch X_B (m rows, d columns, row-major):
+//   pass 1  partial margins: CTA p owns column segments p, p+P, ... of 1024 columns,
+//           keeps its slice of u in registers and writes sum_{cols} x_jc u_c for every
+//           row j to work[(k*P + p)*m + j]   (no atomics, fixed summation order)
+//   pass 2  every CTA sums the P partials of each row, forms the step coefficients
+//           (lr/m) * y_j / (1 + exp(y_j m_j)) in shared memory and updates 512 columns
+//           of u with sum_j coef_j x_jc.  X_B is normally still in L2 for this pass.
+// No tensor cores: with m = 64 rows the work is 64 dot products, bound by memory.
+#include "qesgd_internal.h"
+
+namespace {
+
+constexpr int SEG = 1024;        // columns per segment in pass 1 (32 lanes x 8 float4)
+constexpr int MAX_PARTS = 64;    // partial-margin slots per worker
+constexpr int UPD_THREADS = 128; // pass 2: 4 columns per thread
+
+struct LrArgs {
+    const float *X;
+    uint64_t x_stride;   // elements between workers
+    const float *y;
+    uint64_t y_stride;
+    uint32_t m;
+    uint64_t d;
+    float rate;          // lr / m
+    float *u;
+    uint64_t u_stride;
+    float *work;
+    uint32_t parts;      // P
+    uint32_t nseg;
+};
+
+template <bool VEC>
+__global__ void __launch_bounds__(256) qesgd_lr_margin_kernel(const LrArgs a)
+{
+    __shared__ float s_part[QESGD_MAX_LR_BATCH];
+    const uint32_t lane = threadIdx.x & 31u, warp = threadIdx.x >> 5;
+    const uint32_t k = blockIdx.y, p = blockIdx.x;
+    const float *__restrict__ X = a.X + (uint64_t)k * a.x_stride;
+    const float *__restrict__ u = a.u + (uint64_t)k * a.u_stride;
+    for (uint32_t j = threadIdx.x; j < a.m; j += blockDim.x) s_part[j] = 0.0f;
+    __syncthreads();
+
+    for (uint32_t seg = p; seg < a.nseg; seg += a.parts) {
+        const uint64_t c0 = (uint64_t)seg * SEG;
+        float4 uu[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint64_t c = c0 + (uint64_t)i * 128 + lane * 4u;
+            if (VEC && c + 4 <= a.d) {
+                uu[i] = *reinterpret_cast<const float4 *>(u + c);
+            } else {
+                uu[i].x = c + 0 < a.d ? u[c + 0] : 0.0f;
+                uu[i].y = c + 1 < a.d ? u[c + 1] : 0.0f;
+                uu[i].z = c + 2 < a.d ? u[c + 2] : 0.0f;
+                uu[i].w = c + 3 < a.d ? u[c + 3] : 0.0f;
+            }
+        }
+        for (uint32_t j = warp; j < a.m; j += 8) {  // each row belongs to one warp
+            const float *__restrict__ row = X + (uint64_t)j * a.d;
+            float4 xx[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const uint64_t c = c0 + (uint64_t)i * 128 + lane * 4u;
+                if (VEC && c + 4 <= a.d) {
+                    xx[i] = __ldg(reinterpret_cast<const float4 *>(row + c));
+                } else {
+                    xx[i].x = c + 0 < a.d ? __ldg(row + c + 0) : 0.0f;
+                    xx[i].y = c + 1 < a.d ? __ldg(row + c + 1) : 0.0f;
+                    xx[i].z = c + 2 < a.d ? __ldg(row + c + 2) : 0.0f;
+                    xx[i].w = c + 3 < a.d ? __ldg(row + c + 3) : 0.0f;
+                }
+            }
+            float acc = 0.0f;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                acc = fmaf(xx[i].x, uu[i].x, acc);
+                acc = fmaf(xx[i].y, uu[i].y, acc);
+                acc = fmaf(xx[i].z, uu[i].z, acc);
+                acc = fmaf(xx[i].w, uu[i].w, acc);
+            }
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+            if (lane == 0) s_part[j] += acc;
+        }
+    }
+    __syncthreads();
+    float *__restrict__ out = a.work + ((uint64_t)k * a.parts + p) * a.m;
+    for (uint32_t j = threadIdx.x; j < a.m; j += blockDim.x) out[j] = s_part[j];
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(UPD_THREADS) qesgd_lr_update_kernel(const LrArgs a)
+{
+    __shared__ float s_coef[QESGD_MAX_LR_BATCH];
+    const uint32_t k = blockIdx.y;
+    const float *__restrict__ X = a.X + (uint64_t)k * a.x_stride;
+    const float *__restrict__ y = a.y + (uint64_t)k * a.y_stride;
+    float *__restrict__ u = a.u + (uint64_t)k * a.u_stride;
+    const float *__restrict__ work = a.work + (uint64_t)k * a.parts * a.m;
+    for (uint32_t j = threadIdx.x; j < a.m; j += blockDim.x) {
+        float margin = 0.0f;
+        for (uint32_t p = 0; p < a.parts; ++p) margin += work[(uint64_t)p * a.m + j];
+        const float yj = __ldg(y + j);
+        // -(lr/m) * c_j with c_j = -y_j / (1 + exp(y_j m_j))
+        s_coef[j] = a.rate * yj / (1.0f + expf(yj * margin));
+    }
+    __syncthreads();
+
+    const uint64_t c = ((uint64_t)blockIdx.x * UPD_THREADS + threadIdx.x) * 4u;
+    if (c >= a.d) return;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (VEC && c + 4 <= a.d) {
+        const float *__restrict__ col = X + c;
+#pragma unroll 8
+        for (uint32_t j = 0; j < a.m; ++j) {
+            const float4 x = __ldg(reinterpret_cast<const float4 *>(col + (uint64_t)j * a.d));
+            const float cj = s_coef[j];
+            acc.x = fmaf(cj, x.x, acc.x);
+            acc.y = fmaf(cj, x.y, acc.y);
+            acc.z = fmaf(cj, x.z, acc.z);
+            acc.w = fmaf(cj, x.w, acc.w);
+        }
+        float4 uu = *reinterpret_cast<float4 *>(u + c);
+        uu.x += acc.x; uu.y += acc.y; uu.z += acc.z; uu.w += acc.w;
+        *reinterpret_cast<float4 *>(u + c) = uu;
+    } else {
+        for (int e = 0; e < 4; ++e) {
+            if (c + e >= a.d) break;
+            float s = 0.0f;
+            for (uint32_t j = 0; j < a.m; ++j)
+                s = fmaf(s_coef[j], __ldg(X + (uint64_t)j * a.d + c + e), s);
+            u[c + e] += s;
+        }
+    }
+}
+
+}  // namespace
+
+int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float *yb,
+                         uint64_t y_worker_stride, uint32_t m, uint64_t d, uint32_t K, float lr,
+                         float *u, uint64_t u_stride, float *work, uint64_t work_floats,
+                         cudaStream_t stream, int *launched)
+{
+    *launched = 0;
+    LrArgs a;
+    a.X = Xb; a.x_stride = x_worker_stride;
+    a.y = yb; a.y_stride = y_worker_stride;
+    a.m = m; a.d = d;
+    a.rate = lr / (float)m;
+    a.u = u; a.u_stride = u_stride;
+    a.work = work;
+    const uint64_t nseg = (d + SEG - 1) / SEG;
+    uint64_t parts = work_floats / ((uint64_t)K * m);
+    if (parts > (uint64_t)MAX_PARTS) parts = MAX_PARTS;
+    if (parts > nseg) parts = nseg;
+    if (parts == 0 || nseg > 0xFFFFFFFFull) return (int)cudaErrorInvalidValue;
+    a.parts = (uint32_t)parts;
+    a.nseg = (uint32_t)nseg;
+    const bool vec = (d % 4 == 0) && (x_worker_stride % 4 == 0) && (u_stride % 4 == 0) &&
+                     (((uintptr_t)Xb | (uintptr_t)u) % 16 == 0);
+    dim3 g1((unsigned)parts, K), b1(256);
+    if (vec) qesgd_lr_margin_kernel<true><<<g1, b1, 0, stream>>>(a);
+    else qesgd_lr_margin_kernel<false><<<g1, b1, 0, stream>>>(a);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return (int)e;
+    *launched = 1;
+    const uint64_t ublocks = (d + UPD_THREADS * 4 - 1) / (UPD_THREADS * 4);
+    if (ublocks > 0x7FFFFFFFull) return (int)cudaErrorInvalidValue;
+    dim3 g2((unsigned)ublocks, K), b2(UPD_THREADS);
+    if (vec) qesgd_lr_update_kernel<true><<<g2, b2, 0, stream>>>(a);
+    else qesgd_lr_update_kernel<false><<<g2, b2, 0, stream>>>(a);
+    e = cudaGetLastError();
+    if (e == cudaSuccess) *launched = 2;
+    return (int)e;
+}

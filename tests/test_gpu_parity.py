@@ -1,0 +1,272 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle
+on the same seeded inputs.  Codes and scales must match bit for bit; applied
+parameters within 1e-6 relative; the logistic step within 1e-5 relative."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():
+    pytest.skip("no CUDA device", allow_module_level=True)
+
+from oracle import qesgd_ref as ref                         # noqa: E402
+from paper_1901_03040_b200 import qesgd, synthetic          # noqa: E402
+from tests import gpu_helpers as G                          # noqa: E402
+
+BITS_S = [(2, 1), (4, 7), (4, 5), (8, 127), (8, 100)]
+BUCKETS = [64, 128, 256, 512, 1024, 2048, 4096, 8192]
+
+
+def _delta(n, seed, sigma=1e-3, outliers=True):
+    return synthetic.delta_vector(n, sigma, seed, 0, 0.01 if outliers else 0.0)
+
+
+def _assert_streams_equal(got, want):
+    gc, gs, gst = got
+    wc, ws, wst = want
+    assert gs.dtype == ws.dtype == np.float32
+    bad = np.nonzero(gs.view(np.uint32) != ws.view(np.uint32))[0]
+    assert bad.size == 0, f"{bad.size} scales differ, first bucket {bad[:5]}: {gs[bad[:5]]} vs {ws[bad[:5]]}"
+    badc = np.nonzero(gc != wc)[0]
+    assert badc.size == 0, f"{badc.size} code words differ, first {badc[:5]}"
+    assert gst == wst
+
+
+# ----------------------------------------------------------------- encode ----
+@pytest.mark.parametrize("mode", [ref.SCALE_NORM, ref.SCALE_MAX])
+@pytest.mark.parametrize("bucket", BUCKETS)
+@pytest.mark.parametrize("bits,s", BITS_S)
+def test_encode_matches_oracle_bitwise(bits, s, bucket, mode):
+    # several CTA tiles, a ragged tail that is neither a multiple of 8 nor of the bucket
+    n = 8192 * 3 + 1000 + 3
+    z = _delta(n, seed=bucket + bits)
+    args = (bucket, s, bits, mode, 0x1234_5678_9ABC_DEF0, 3, 17)
+    _assert_streams_equal(G.gpu_encode(z, None, *args), ref.encode(z, None, *args))
+
+
+@pytest.mark.parametrize("n", [1, 7, 8, 63, 64, 65, 511, 512, 513, 4095, 8193])
+@pytest.mark.parametrize("bucket", [64, 512, 4096])
+def test_encode_small_and_ragged_sizes(n, bucket):
+    z = _delta(n, seed=n)
+    w = synthetic.anchor_vector(n, seed=n + 1)
+    u = (w + z).astype(np.float32)
+    for mode in (ref.SCALE_NORM, ref.SCALE_MAX):
+        args = (bucket, 7, 4, mode, 99, 1, 2)
+        _assert_streams_equal(G.gpu_encode(u, w, *args), ref.encode(u, w, *args))
+
+
+@pytest.mark.parametrize("bits,s", [(2, 1), (4, 7), (8, 127)])
+def test_encode_with_anchor_large(bits, s):
+    n = (1 << 20) + 40
+    w = synthetic.anchor_vector(n, seed=5)
+    u = (w + _delta(n, seed=6, sigma=1e-4)).astype(np.float32)
+    args = (512, s, bits, ref.SCALE_NORM, 7, 0, 0)
+    _assert_streams_equal(G.gpu_encode(u, w, *args), ref.encode(u, w, *args))
+
+
+def test_encode_unaligned_pointer_takes_the_scalar_path():
+    n = 8192 + 77
+    z = _delta(n, seed=31)
+    args = (256, 7, 4, ref.SCALE_NORM, 5, 0, 1)
+    want = ref.encode(z, None, *args)
+    for mis in (1, 3, 4):
+        _assert_streams_equal(G.gpu_encode(z, None, *args, misalign=mis), want)
+
+
+def test_encode_batch_uses_worker_ids_and_strides():
+    K, n, bucket = 5, 8192 + 520, 128
+    w = synthetic.anchor_vector(n, seed=1)
+    locs = synthetic.worker_locals(w, K, 1e-4, seed=2)
+    gc, gs, gst = G.gpu_encode_batch(locs, w, bucket, 7, 4, ref.SCALE_NORM, 42, 10, 3)
+    assert gst == 0
+    for k in range(K):
+        wc, ws, _ = ref.encode(locs[k], w, bucket, 7, 4, ref.SCALE_NORM, 42, 10 + k, 3)
+        assert (gc[k] == wc).all() and (gs[k].view(np.uint32) == ws.view(np.uint32)).all()
+
+
+def test_encode_epoch_and_seed_change_the_draws_but_not_the_scales():
+    z = _delta(4096, seed=8)
+    a = G.gpu_encode(z, None, 512, 7, 4, ref.SCALE_NORM, 1, 0, 0)
+    b = G.gpu_encode(z, None, 512, 7, 4, ref.SCALE_NORM, 1, 0, 1)
+    c = G.gpu_encode(z, None, 512, 7, 4, ref.SCALE_NORM, 1, 0, 0)
+    assert (a[0] == c[0]).all() and (a[0] != b[0]).any() and (a[1] == b[1]).all()
+
+
+@pytest.mark.parametrize("mode", [ref.SCALE_NORM, ref.SCALE_MAX])
+def test_nonfinite_zero_tiny_and_huge_buckets(mode):
+    n = 64 * 8
+    z = _delta(n, seed=3)
+    z[70] = np.inf
+    z[130] = np.nan
+    z[192:256] = 0.0
+    z[256:320] = np.float32(2.0 ** -120)
+    z[320:384] = np.float32(3e38)
+    z[384:448] = np.float32(1e-42)        # subnormal inputs
+    z[448] = -np.inf
+    args = (64, 7, 4, mode, 11, 0, 0)
+    got, want = G.gpu_encode(z, None, *args), ref.encode(z, None, *args)
+    _assert_streams_equal(got, want)
+    assert got[2] == qesgd.STATUS_NONFINITE
+    assert G.ctx().qesgd_status() == 0            # reading the status clears it
+
+
+def test_subnormal_and_mixed_magnitudes_match():
+    rng = np.random.default_rng(12)
+    n = 4096
+    z = (rng.standard_normal(n) * np.exp(rng.uniform(-80, 20, n))).astype(np.float32)
+    for bucket in (64, 1024):
+        for mode in (ref.SCALE_NORM, ref.SCALE_MAX):
+            args = (bucket, 127, 8, mode, 2, 1, 1)
+            _assert_streams_equal(G.gpu_encode(z, None, *args), ref.encode(z, None, *args))
+
+
+def test_fixed_delta_mode_matches_and_clips():
+    n = 8192 + 100
+    z = _delta(n, seed=21)
+    z[5] = np.nan
+    z[9] = np.inf
+    z[10] = -np.inf
+    delta = 2.5e-4
+    for bits, s in ((4, 7), (8, 127), (2, 1)):
+        got = G.gpu_encode(z, None, 512, s, bits, ref.SCALE_FIXED, 3, 2, 1, fixed_delta=delta)
+        want = ref.encode(z, None, 512, s, bits, ref.SCALE_FIXED, 3, 2, 1, fixed_delta=delta)
+        _assert_streams_equal(got, want)
+        assert got[2] == qesgd.STATUS_NONFINITE
+
+
+def test_on_grid_input_round_trips_exactly_on_the_gpu():
+    s, bits, bucket = 127, 8, 256
+    rng = np.random.default_rng(4)
+    n = bucket * 40
+    k = rng.integers(-s, s + 1, n)
+    k[::bucket] = s
+    z = (k * 2.0 ** -14).astype(np.float32)
+    codes, scales, status = G.gpu_encode(z, None, bucket, s, bits, ref.SCALE_MAX, 77, 0, 0)
+    assert status == 0 and (scales == np.float32(s * 2.0 ** -14)).all()
+    assert (G.gpu_decode(codes, scales, n, bucket, s, bits) == z).all()
+
+
+# ----------------------------------------------------------------- decode ----
+@pytest.mark.parametrize("bucket", [64, 512, 8192])
+@pytest.mark.parametrize("bits,s", BITS_S)
+def test_decode_matches_oracle_bitwise(bits, s, bucket):
+    n = 8192 * 2 + 333
+    z = _delta(n, seed=bits * 100 + s)
+    codes, scales, _ = ref.encode(z, None, bucket, s, bits, ref.SCALE_NORM, 9, 0, 0)
+    got = G.gpu_decode(codes, scales, n, bucket, s, bits)
+    want = ref.decode(codes, scales, n, bucket, s, bits)
+    assert (got.view(np.uint32) == want.view(np.uint32)).all()
+
+
+# --------------------------------------------------- decode-average-apply ----
+def _daa_case(n, K, bucket, bits, s, seed, sigma=1e-4):
+    w = synthetic.anchor_vector(n, seed=seed)
+    locs = synthetic.worker_locals(w, K, sigma, seed=seed + 1, outlier_prob=0.01)
+    codes, scales = [], []
+    for k in range(K):
+        c, sc, _ = ref.encode(locs[k], w, bucket, s, bits, ref.SCALE_NORM, seed, k, 0)
+        codes.append(c)
+        scales.append(sc)
+    return w, np.stack(codes), np.stack(scales)
+
+
+def _assert_param_close(got, want, w_before, scales, bucket):
+    smax = np.repeat(scales.max(axis=0), bucket)[:want.size]
+    tol = 1e-6 * np.maximum(np.abs(want), smax)
+    err = np.abs(got.astype(np.float64) - want.astype(np.float64))
+    assert (err <= tol).all(), f"max err/tol {np.max(err / np.maximum(tol, 1e-300))}"
+    assert (got != w_before).any()
+
+
+@pytest.mark.parametrize("K", [1, 2, 3, 8, 16, 33, 64])
+@pytest.mark.parametrize("bucket,bits,s", [(64, 4, 7), (128, 2, 1), (256, 2, 1), (512, 4, 7),
+                                           (2048, 8, 127), (8192, 4, 7)])
+def test_decode_average_apply_matches_oracle(K, bucket, bits, s):
+    n = 8192 * 2 + 300 + 5
+    w, codes, scales = _daa_case(n, K, bucket, bits, s, seed=K * 7 + bits)
+    got = G.gpu_decode_average_apply(w, codes, scales, bucket, s, bits)
+    want = ref.decode_average_apply(w, codes, scales, bucket, s, bits)
+    _assert_param_close(got, want, w, scales, bucket)
+
+
+@pytest.mark.parametrize("n", [1, 9, 255, 256, 257, 2049])
+def test_decode_average_apply_small_sizes(n):
+    w, codes, scales = _daa_case(n, 4, 64, 4, 7, seed=n)
+    got = G.gpu_decode_average_apply(w, codes, scales, 64, 7, 4)
+    want = ref.decode_average_apply(w, codes, scales, 64, 7, 4)
+    _assert_param_close(got, want, w, scales, 64)
+
+
+def test_k1_on_grid_apply_returns_the_worker_parameter_exactly():
+    rng = np.random.default_rng(6)
+    n, s, bits, bucket = 512 * 9, 127, 8, 512
+    k = rng.integers(-s, s + 1, n)
+    k[::bucket] = s
+    z = (k * 2.0 ** -10).astype(np.float32)
+    w = (rng.integers(-1000, 1000, n) * 2.0 ** -10).astype(np.float32)
+    codes, scales, _ = G.gpu_encode(w + z, w, bucket, s, bits, ref.SCALE_MAX, 1, 0, 0)
+    out = G.gpu_decode_average_apply(w, codes[None], scales[None], bucket, s, bits)
+    assert (out == w + z).all()
+
+
+# ----------------------------------------------------- logistic regression ---
+def _lr_close(got, want):
+    dn = np.linalg.norm(got.astype(np.float64) - want)
+    assert dn <= 1e-5 * np.linalg.norm(want)
+    assert np.abs(got - want).max() <= 1e-5 * np.abs(want).max()
+
+
+@pytest.mark.parametrize("m,d", [(64, 4096), (64, 65536), (7, 1000), (1, 5), (200, 3001),
+                                 (1024, 2048)])
+def test_lr_step_matches_oracle(m, d):
+    X, y, _ = synthetic.logistic_problem(m, d, seed=m + d)
+    u = (0.3 * synthetic.normal_f32(d, 1.0, 5)).astype(np.float32)
+    tu = G.dev(u)
+    G.ctx().qesgd_lr_sgd_step(G.dev(X), G.dev(y), m, d, 0.1, tu)
+    _lr_close(tu.cpu().numpy(), ref.lr_sgd_step(X, y, 0.1, u))
+
+
+def test_lr_local_epoch_and_batch_match_oracle():
+    K, n_local, d, batch = 3, 150, 2048, 64
+    X, y, _ = synthetic.logistic_problem(K * n_local, d, seed=9)
+    u0 = np.zeros(d, dtype=np.float32)
+    tu = torch.zeros((K, d), dtype=torch.float32, device="cuda")
+    G.ctx().qesgd_lr_local_epoch_batch(G.dev(X), G.dev(y), n_local, d, K, batch, 0.5, tu, d)
+    got = tu.cpu().numpy()
+    for k in range(K):
+        rows = slice(k * n_local, (k + 1) * n_local)
+        want = ref.lr_local_epoch(X[rows], y[rows], batch, 0.5, u0)
+        _lr_close(got[k], want)
+    t1 = torch.zeros(d, dtype=torch.float32, device="cuda")
+    G.ctx().qesgd_lr_local_epoch(G.dev(X[:n_local]), G.dev(y[:n_local]), n_local, d, batch, 0.5, t1)
+    assert (t1.cpu().numpy() == got[0]).all()
+
+
+# ------------------------------------------------------ argument checking ----
+def test_invalid_arguments_return_einval_and_launch_nothing():
+    c = G.ctx()
+    z = torch.zeros(4096, device="cuda")
+    codes, scales = qesgd.alloc_stream_buffers(1, 4096, 512, 4, "cuda")
+    before = c.qesgd_launch_count()
+    bad = [dict(bucket=48), dict(bucket=16384), dict(bits=3), dict(s=8), dict(s=0), dict(mode=3)]
+    for kw in bad:
+        a = dict(bucket=512, s=7, bits=4, mode=0)
+        a.update(kw)
+        with pytest.raises(qesgd.QesgdError) as ei:
+            c.qesgd_encode(z, None, 4096, a["bucket"], a["s"], a["bits"], a["mode"], 0, 0, 0,
+                           codes, scales)
+        assert ei.value.code == qesgd.EINVAL
+    with pytest.raises(qesgd.QesgdError):
+        c.qesgd_encode(z, None, 4096, 512, 7, 4, qesgd.SCALE_FIXED, 0, 0, 0, codes, scales,
+                       fixed_delta=0.0)
+    with pytest.raises(qesgd.QesgdError):
+        c.qesgd_encode(None, None, 4096, 512, 7, 4, 0, 0, 0, 0, codes, scales)
+    with pytest.raises(qesgd.QesgdError):
+        c.qesgd_decode_average_apply(z, 4096, 65, codes, 0, scales, 0, 512, 7, 4)
+    with pytest.raises(qesgd.QesgdError):
+        c.qesgd_encode(z, None, 4096, 512, 7, 4, 0, 0, 0, 0, codes.view(-1)[4:], scales)
+    c.qesgd_encode(z, None, 0, 512, 7, 4, 0, 0, 0, 0, codes, scales)      # d = 0: no-op
+    c.qesgd_decode_average_apply(z, 0, 3, codes, 0, scales, 0, 512, 7, 4)
+    assert c.qesgd_launch_count() == before
+    assert c.qesgd_status() == 0
