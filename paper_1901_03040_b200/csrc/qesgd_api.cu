@@ -152,6 +152,7 @@ int qesgd_encode_batch(qesgd_ctx *ctx, const float *local, uint64_t local_stride
     a.key1 = (uint32_t)(seed >> 32);
     a.worker0 = worker0;
     a.epoch = epoch;
+    a.K = K;
     a.codes = codes_out;
     a.code_stride = K > 1 ? code_stride : 0;
     a.scales = scales_out;

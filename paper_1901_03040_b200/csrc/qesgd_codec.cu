@@ -120,10 +120,13 @@ __global__ void __launch_bounds__(256) qesgd_encode_kernel(const EncodeArgs a)
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
     const uint32_t warps = blockDim.x >> 5;
-    const uint32_t k = blockIdx.y;
+    // Workers vary fastest over the grid: the K CTAs that share a tile of the anchor run
+    // close together in time, so the anchor comes from HBM once and from L2 K-1 times.
+    const uint32_t k = blockIdx.x % a.K;
+    const uint32_t tile = blockIdx.x / a.K;
     const uint32_t lb = a.log2_bucket;
     const float *__restrict__ local = a.local + (uint64_t)k * a.local_stride;
-    const uint64_t warp_base = ((uint64_t)blockIdx.x * warps + warp) * (uint64_t)(V * CHUNK);
+    const uint64_t warp_base = ((uint64_t)tile * warps + warp) * (uint64_t)(V * CHUNK);
 
     // ---- loads: everything this lane needs is requested before any use -------
     float z[V][8];
@@ -428,8 +431,8 @@ cudaError_t launch_encode_v(const EncodeArgs &a, uint32_t K, cudaStream_t stream
     static_assert(warps * V * CHUNK >= QESGD_MAX_BUCKET, "a bucket never leaves its CTA");
     const uint64_t tile = (uint64_t)warps * V * CHUNK;
     const uint64_t tiles = (a.padded + tile - 1) / tile;
-    if (tiles == 0 || tiles > 0x7FFFFFFFull) return cudaErrorInvalidValue;
-    dim3 grid((unsigned)tiles, K, 1), block(warps * 32u, 1, 1);
+    if (tiles == 0 || tiles * K > 0x7FFFFFFFull) return cudaErrorInvalidValue;
+    dim3 grid((unsigned)(tiles * K), 1, 1), block(warps * 32u, 1, 1);
     qesgd_encode_kernel<BITS, MODE, ANCHOR, VEC, V><<<grid, block, 0, stream>>>(a);
     return cudaGetLastError();
 }

@@ -32,6 +32,7 @@ struct EncodeArgs {
     float fixed_scale;      // fl32(s * delta), FIXED mode only
     uint32_t key0, key1;    // seed low / high
     uint32_t worker0, epoch;
+    uint32_t K;             // workers in this launch
     uint32_t *codes;
     uint64_t code_stride;   // bytes between workers
     float *scales;
