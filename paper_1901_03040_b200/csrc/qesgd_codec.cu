@@ -80,53 +80,158 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 
 // ------------------------------------------------------- rounding (Eq. 4) ----
 // level = floor(r) + [h + 1/2 < frac(r) * 2^16] for r = min(|z|*inv, s), 0 <= r <= 127.
-// Adding 2^23 with round-toward-zero leaves 2^23 + floor(r) in the mantissa, which
-// gives floor(r) both as a float (one exact subtract) and as the low byte of the bit
-// pattern; (2^23 + h) - (2^23 - 1/2) is h + 1/2 exactly.  All full-rate fp32/int ops.
-__device__ __forceinline__ uint32_t stochastic_level(float a, float inv, float sf, uint32_t h)
+//
+// With U = ceil(r * 2^16 - 1/2) the level is (U + 65535 - h) >> 16: writing U =
+// floor(r) * 2^16 + T, T = ceil(frac(r) * 2^16 - 1/2) in [0, 2^16], the draw rounds
+// up iff h < T.  U comes from ONE fused multiply-add rounded toward +infinity:
+// r * 2^16 + (2^23 - 1/2) lies in [2^23, 2^24) where floats are the integers, so
+// the bit pattern of the result is 0x4B000000 + U.  r is kept >= 2^-30 so that
+// r = 0 (where the sum would be 2^23 - 1/2 exactly, below the integer binade)
+// gives U = 0 like every r with r * 2^16 <= 1/2; the same clamp turns the NaN of
+// an invalid bucket (inv = 0) into level 0.
+__device__ __forceinline__ uint32_t level_times_65536(float a, float inv, float sf, uint32_t h)
 {
-    const float r = fminf(__fmul_rn(a, inv), sf);
-    const float t = __fadd_rz(r, 8388608.0f);
-    const float f = __fsub_rn(t, 8388608.0f);
-    const float p = __fsub_rn(r, f);
-    const float hh = __fsub_rn(__uint_as_float(0x4B000000u | h), 8388607.5f);
-    const uint32_t up = hh < __fmul_rn(p, 65536.0f) ? 1u : 0u;
-    return (__float_as_uint(t) & 0xFFu) + up;
+    const float r = fminf(fmaxf(__fmul_rn(a, inv), 0x1p-30f), sf);
+    const uint32_t ub = __float_as_uint(__fmaf_ru(r, 65536.0f, 8388607.5f));
+    return ub - h + (65535u - 0x4B000000u);   // level in bits 16..22, below: don't care
 }
 
-// code = sign << (BITS-1) | level with no "-0" code; returned already shifted to slot j.
-template <int BITS>
-__device__ __forceinline__ uint32_t place_code(uint32_t level, uint32_t zbits, int slot)
+// Packing.  X[j] holds the level of element j in byte 2 (bits 16..22) and Z[j] the
+// sign of z_j in bit 31.  Bytes are gathered with PRMT, fields merged with
+// multiply-adds; the sign is kept only where the level is not zero, which is
+// tested on whole words (a field plus its largest level never carries).
+__device__ __forceinline__ uint32_t bytes2(uint32_t a, uint32_t b)   // [a.b2, b.b2, 0, 0]
 {
-    // bit 31 of (level + 0x7FFFFFFF) is set iff level > 0
-    const uint32_t sign31 = zbits & (level + 0x7FFFFFFFu) & 0x80000000u;
-    const int top = slot * BITS + BITS - 1;
-    return (level << (slot * BITS)) | (sign31 >> (31 - top));
+    return __byte_perm(a, b, 0x0062) & 0xFFFFu;
+}
+__device__ __forceinline__ uint32_t bytes3(uint32_t a, uint32_t b)   // [a.b3, b.b3, ., .]
+{
+    return __byte_perm(a, b, 0x0073);
+}
+
+template <int BITS>
+__device__ __forceinline__ void pack_octet(const uint32_t (&X)[8], const uint32_t (&Z)[8],
+                                           uint32_t (&out)[2])
+{
+    if (BITS == 8) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int e = 4 * h;
+            const uint32_t lv = __byte_perm(__byte_perm(X[e], X[e + 1], 0x0062),
+                                            __byte_perm(X[e + 2], X[e + 3], 0x0062), 0x5410);
+            const uint32_t sg = __byte_perm(bytes3(Z[e], Z[e + 1]), bytes3(Z[e + 2], Z[e + 3]), 0x5410);
+            out[h] = lv | (sg & (lv + 0x7F7F7F7Fu) & 0x80808080u);
+        }
+    } else if (BITS == 4) {
+        // even elements fill the low nibbles, odd elements the high nibbles
+        const uint32_t le = __byte_perm(__byte_perm(X[0], X[2], 0x0062), __byte_perm(X[4], X[6], 0x0062), 0x5410);
+        const uint32_t lo = __byte_perm(__byte_perm(X[1], X[3], 0x0062), __byte_perm(X[5], X[7], 0x0062), 0x5410);
+        const uint32_t lv = le + lo * 16u;
+        const uint32_t se = __byte_perm(bytes3(Z[0], Z[2]), bytes3(Z[4], Z[6]), 0x5410);
+        const uint32_t so = __byte_perm(bytes3(Z[1], Z[3]), bytes3(Z[5], Z[7]), 0x5410);
+        const uint32_t sg = ((se >> 4) & 0x08080808u) | (so & 0x80808080u);
+        out[0] = lv | (sg & (lv + 0x77777777u));
+        out[1] = 0u;
+    } else {
+        // element j sits at bits 2j, 2j+1: byte 0 holds elements 0..3, byte 1 elements 4..7
+        const uint32_t g0 = bytes2(X[0], X[4]), g1 = bytes2(X[1], X[5]);
+        const uint32_t g2 = bytes2(X[2], X[6]), g3 = bytes2(X[3], X[7]);
+        const uint32_t lv = (g0 + g1 * 4u) + (g2 * 16u + g3 * 64u);
+        const uint32_t h0 = bytes3(Z[0], Z[4]), h1 = bytes3(Z[1], Z[5]);
+        const uint32_t h2 = bytes3(Z[2], Z[6]), h3 = bytes3(Z[3], Z[7]);
+        const uint32_t sg = ((h0 >> 6) & 0x0202u) | ((h1 >> 4) & 0x0808u) | ((h2 >> 2) & 0x2020u) |
+                            (h3 & 0x8080u);
+        out[0] = lv | (sg & (lv << 1));
+        out[1] = 0u;
+    }
+}
+
+// ----------------------------------------------------- bucket reductions ----
+struct SumF64 {
+    typedef double T;
+    static __device__ __forceinline__ double op(double x, double y) { return __dadd_rn(x, y); }
+};
+struct MaxU32 {
+    typedef uint32_t T;
+    static __device__ __forceinline__ uint32_t op(uint32_t x, uint32_t y) { return max(x, y); }
+};
+
+// Reduces the four per-chunk partials of every lane over the lanes (and chunks) of a
+// bucket, in the order of the balanced binary tree on element index: lanes xor 1, 2,
+// 4, (8), (16), then chunk pairs, then chunk quads.  The first two steps hand each
+// lane ONE chunk to carry on with (even/odd lanes split chunks {0,1}/{2,3}, then bit 1
+// of the lane splits the pair), so the rest of the tree costs one value per step
+// instead of four.  On return lane L holds the bucket total of chunk
+// 2*(L&1) + ((L>>1)&1) of its own lane group (for buckets >= 512 the chunks of one
+// bucket all hold its total).
+template <typename R>
+__device__ __forceinline__ typename R::T reduce_chunks(const typename R::T (&t)[4], uint32_t lane,
+                                                       uint32_t lb)
+{
+    typedef typename R::T T;
+    const bool b0 = lane & 1u, b1 = lane & 2u;
+    T k0 = b0 ? t[2] : t[0], k1 = b0 ? t[3] : t[1];
+    const T s0 = b0 ? t[0] : t[2], s1 = b0 ? t[1] : t[3];
+    k0 = R::op(k0, __shfl_xor_sync(FULL, s0, 1));
+    k1 = R::op(k1, __shfl_xor_sync(FULL, s1, 1));
+    T k = b1 ? k1 : k0;
+    const T s = b1 ? k0 : k1;
+    k = R::op(k, __shfl_xor_sync(FULL, s, 2));
+    k = R::op(k, __shfl_xor_sync(FULL, k, 4));
+    if (lb >= 7) k = R::op(k, __shfl_xor_sync(FULL, k, 8));
+    if (lb >= 8) k = R::op(k, __shfl_xor_sync(FULL, k, 16));
+    if (lb >= 9) k = R::op(k, __shfl_xor_sync(FULL, k, 2));    // chunks (0,1) and (2,3)
+    if (lb >= 10) k = R::op(k, __shfl_xor_sync(FULL, k, 1));   // all four chunks
+    return k;
+}
+
+// Buckets wider than a warp's 1024 elements: combine the totals of the wpb = bucket/1024
+// consecutive warps that share a bucket, adjacent pairs first.
+template <typename R>
+__device__ __forceinline__ typename R::T reduce_warps(typename R::T k, typename R::T *smem,
+                                                      uint32_t lane, uint32_t warp, uint32_t lb)
+{
+    typedef typename R::T T;
+    const uint32_t wpb = 1u << (lb - 10);
+    if (lane == 0) smem[warp] = k;
+    __syncthreads();
+    const uint32_t g0 = warp & ~(wpb - 1u);
+    T acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = smem[(g0 + i) & 7u];
+#pragma unroll
+    for (int w2 = 1; w2 < 8; w2 <<= 1) {
+        if ((uint32_t)w2 < wpb) {
+#pragma unroll
+            for (int i = 0; i < 8; i += 2 * w2) acc[i] = R::op(acc[i], acc[i + w2]);
+        }
+    }
+    return acc[0];
 }
 
 // ------------------------------------------------------------- encode -------
 // MODE: 0 = L2 norm, 1 = max magnitude, 2 = caller-given spacing.
-// V = chunks per warp; a warp owns V*256 consecutive elements, a CTA of W warps
-// owns W*V*256.  Buckets are powers of two in [64, 8192]:
-//   bucket <= 256      : bucket/8 lanes of one chunk
-//   bucket <= 256*V    : bucket/256 chunks of one warp
-//   bucket  > 256*V    : bucket/(256*V) consecutive warps of the CTA (shared memory)
-template <int BITS, int MODE, bool ANCHOR, bool VEC, int V>
+// A warp owns V = 4 chunks = 1024 consecutive elements, a CTA of 8 warps 8192.
+// Buckets are powers of two in [64, 8192]:
+//   bucket <= 256   : bucket/8 lanes of one chunk
+//   bucket <= 1024  : bucket/256 chunks of one warp
+//   bucket  > 1024  : bucket/1024 consecutive warps of the CTA (shared memory)
+template <int BITS, int MODE, bool ANCHOR, bool VEC>
 __global__ void __launch_bounds__(256) qesgd_encode_kernel(const EncodeArgs a)
 {
+    constexpr int V = 4;
     __shared__ double s_part[8];
     __shared__ uint32_t s_max[8];
 
     const uint32_t lane = threadIdx.x & 31u;
     const uint32_t warp = threadIdx.x >> 5;
-    const uint32_t warps = blockDim.x >> 5;
     // Workers vary fastest over the grid: the K CTAs that share a tile of the anchor run
     // close together in time, so the anchor comes from HBM once and from L2 K-1 times.
     const uint32_t k = blockIdx.x % a.K;
     const uint32_t tile = blockIdx.x / a.K;
     const uint32_t lb = a.log2_bucket;
     const float *__restrict__ local = a.local + (uint64_t)k * a.local_stride;
-    const uint64_t warp_base = ((uint64_t)tile * warps + warp) * (uint64_t)(V * CHUNK);
+    const uint64_t warp_base = ((uint64_t)tile * 8u + warp) * (uint64_t)(V * CHUNK);
 
     // ---- loads: everything this lane needs is requested before any use -------
     float z[V][8];
@@ -144,13 +249,13 @@ __global__ void __launch_bounds__(256) qesgd_encode_kernel(const EncodeArgs a)
             for (int j = 0; j < 8; ++j) z[c][j] = __fsub_rn(z[c][j], w[c][j]);
     }
 
-    // ---- per-bucket scale ------------------------------------------------------
-    float scale[V];
-    bool nonfinite[V];
+    // ---- per-bucket scale: one value per lane, then handed back per chunk ------
+    const float sf = (float)a.s;
+    float my_scale, my_inv;
+    bool flag = false;
     if (MODE == 0) {
-        // fp64 sum of squares over the balanced binary tree on index order: 8 in the
-        // lane, then lanes (xor 1,2,4,8,16), then chunks, then warps.  The product of
-        // two fp32 values is exact in fp64, so fma(z1,z1,z0*z0) is fl64(q0+q1).
+        // fp64 sum of squares over the balanced binary tree on index order.  The product
+        // of two fp32 values is exact in fp64, so fma(z1,z1,z0*z0) is fl64(q0+q1).
         double t[V];
 #pragma unroll
         for (int c = 0; c < V; ++c) {
@@ -162,42 +267,9 @@ __global__ void __launch_bounds__(256) qesgd_encode_kernel(const EncodeArgs a)
             }
             t[c] = __dadd_rn(__dadd_rn(q[0], q[1]), __dadd_rn(q[2], q[3]));
         }
-#pragma unroll
-        for (int off = 1; off <= 16; off <<= 1) {
-            if ((uint32_t)(off * 8) < (1u << lb)) {  // partner lane is in the same bucket
-#pragma unroll
-                for (int c = 0; c < V; ++c)
-                    t[c] = __dadd_rn(t[c], __shfl_xor_sync(FULL, t[c], off));
-            }
-        }
-        if (lb >= 9) {
-#pragma unroll
-            for (int c = 0; c < V; c += 2) t[c] = t[c + 1] = __dadd_rn(t[c], t[c + 1]);
-        }
-        if (V == 4 && lb >= 10) t[0] = t[1] = t[2] = t[3] = __dadd_rn(t[0], t[2]);
-        if ((1u << lb) > (uint32_t)(V * CHUNK)) {
-            const uint32_t wpb = (1u << lb) / (uint32_t)(V * CHUNK);  // warps per bucket
-            if (lane == 0) s_part[warp] = t[0];
-            __syncthreads();
-            const uint32_t g0 = warp & ~(wpb - 1u);
-            double acc[8];
-#pragma unroll
-            for (int i = 0; i < 8; ++i) acc[i] = (i < (int)wpb) ? s_part[g0 + i] : 0.0;
-#pragma unroll
-            for (int w2 = 1; w2 < 8; w2 <<= 1) {
-                if ((uint32_t)w2 < wpb) {
-#pragma unroll
-                    for (int i = 0; i < 8; i += 2 * w2) acc[i] = __dadd_rn(acc[i], acc[i + w2]);
-                }
-            }
-#pragma unroll
-            for (int c = 0; c < V; ++c) t[c] = acc[0];
-        }
-#pragma unroll
-        for (int c = 0; c < V; ++c) {
-            scale[c] = __double2float_rn(__dsqrt_rn(t[c]));
-            nonfinite[c] = !(fabsf(scale[c]) <= 3.402823466e38f);  // Inf or NaN
-        }
+        double tot = reduce_chunks<SumF64>(t, lane, lb);
+        if (lb > 10) tot = reduce_warps<SumF64>(tot, s_part, lane, warp, lb);
+        my_scale = __double2float_rn(__dsqrt_rn(tot));
     } else if (MODE == 1) {
         // Largest magnitude: bit patterns of |z| order like unsigned integers, and
         // Inf/NaN patterns compare above every finite value.
@@ -208,89 +280,59 @@ __global__ void __launch_bounds__(256) qesgd_encode_kernel(const EncodeArgs a)
 #pragma unroll
             for (int j = 0; j < 8; ++j) m[c] = max(m[c], __float_as_uint(z[c][j]) & 0x7FFFFFFFu);
         }
-#pragma unroll
-        for (int off = 1; off <= 16; off <<= 1) {
-            if ((uint32_t)(off * 8) < (1u << lb)) {
-#pragma unroll
-                for (int c = 0; c < V; ++c) m[c] = max(m[c], __shfl_xor_sync(FULL, m[c], off));
-            }
-        }
-        if (lb >= 9) {
-#pragma unroll
-            for (int c = 0; c < V; c += 2) m[c] = m[c + 1] = max(m[c], m[c + 1]);
-        }
-        if (V == 4 && lb >= 10) m[0] = m[1] = m[2] = m[3] = max(m[0], m[2]);
-        if ((1u << lb) > (uint32_t)(V * CHUNK)) {
-            const uint32_t wpb = (1u << lb) / (uint32_t)(V * CHUNK);
-            if (lane == 0) s_max[warp] = m[0];
-            __syncthreads();
-            const uint32_t g0 = warp & ~(wpb - 1u);
-            uint32_t mm = 0u;
-            for (uint32_t i = 0; i < wpb; ++i) mm = max(mm, s_max[g0 + i]);
-#pragma unroll
-            for (int c = 0; c < V; ++c) m[c] = mm;
-        }
-#pragma unroll
-        for (int c = 0; c < V; ++c) {
-            nonfinite[c] = m[c] >= 0x7F800000u;
-            scale[c] = __uint_as_float(m[c]);
-        }
+        uint32_t mm = reduce_chunks<MaxU32>(m, lane, lb);
+        if (lb > 10) mm = reduce_warps<MaxU32>(mm, s_max, lane, warp, lb);
+        my_scale = __uint_as_float(mm);
     } else {
-#pragma unroll
-        for (int c = 0; c < V; ++c) {
-            scale[c] = a.fixed_scale;
-            nonfinite[c] = !(fabsf(scale[c]) <= 3.402823466e38f);
-        }
+        my_scale = a.fixed_scale;
+    }
+    {
+        const bool nonfinite = !(my_scale <= 3.402823466e38f);   // Inf or NaN (scales are >= 0)
+        const bool ok = !nonfinite && my_scale >= 0x1p-100f;
+        my_inv = ok ? __fdiv_rn(sf, my_scale) : 0.0f;
+        my_scale = ok ? my_scale : 0.0f;
+        // Lanes past the padded length hold zeros, so a set flag always belongs to real data.
+        flag = nonfinite;
     }
 
     // ---- rounding, packing, stores ---------------------------------------------
-    const float sf = (float)a.s;
     uint8_t *__restrict__ codes = reinterpret_cast<uint8_t *>(a.codes) + (uint64_t)k * a.code_stride;
     float *__restrict__ scales = a.scales + (uint64_t)k * a.scale_stride;
     const uint32_t bucket_mask = (1u << lb) - 1u;
-    bool flag = false;
 
 #pragma unroll
     for (int c = 0; c < V; ++c) {
         const uint64_t eb = warp_base + (uint64_t)c * CHUNK + lane * 8u;
-        const bool ok = !nonfinite[c] && scale[c] >= 0x1p-100f;
-        const float inv = ok ? __fdiv_rn(sf, scale[c]) : 0.0f;
-        if (eb < a.padded && ((uint32_t)eb & bucket_mask) == 0u) {
-            scales[eb >> lb] = ok ? scale[c] : 0.0f;
-            flag |= nonfinite[c];
+        float scale = my_scale, inv = my_inv;
+        if (MODE != 2) {   // chunk c's bucket total sits in the lane of this quad with bits (c>>1, c&1)
+            const int src = (lane & 28u) | ((c >> 1) & 1) | ((c & 1) << 1);
+            scale = __shfl_sync(FULL, my_scale, src);
+            inv = __shfl_sync(FULL, my_inv, src);
         }
+        if (eb < a.padded && ((uint32_t)eb & bucket_mask) == 0u) scales[eb >> lb] = scale;
+
         uint32_t x[4];
         const uint64_t blk = eb >> 3;
         philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.worker0 + k, a.epoch, a.key0, a.key1, x);
 
-        uint32_t word[(8 * BITS) / 32 > 0 ? (8 * BITS) / 32 : 1];
-#pragma unroll
-        for (int i = 0; i < (int)(sizeof(word) / 4); ++i) word[i] = 0u;
-        bool nan_seen = false;
+        uint32_t X[8], Z[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             const uint32_t h = (j & 1) ? (x[j >> 1] >> 16) : (x[j >> 1] & 0xFFFFu);
-            const uint32_t zb = __float_as_uint(z[c][j]);
-            float av = fabsf(z[c][j]);
-            if (MODE == 2) {  // per element: NaN is flagged and encoded as 0, Inf clips
-                const bool isn = (zb & 0x7FFFFFFFu) > 0x7F800000u;
-                nan_seen |= isn;
-                av = isn ? 0.0f : av;
-            }
-            const uint32_t level = stochastic_level(av, inv, sf, h);
-            constexpr int PER_WORD = 32 / BITS;
-            word[j / PER_WORD] |= place_code<BITS>(level, zb, j % PER_WORD);
+            Z[j] = __float_as_uint(z[c][j]);
+            if (MODE == 2)   // NaN has no place on the grid: flagged (and encoded as 0 by the clamp)
+                flag |= (Z[j] & 0x7FFFFFFFu) > 0x7F800000u;
+            X[j] = level_times_65536(fabsf(z[c][j]), inv, sf, h);
         }
-        if (MODE == 2) flag |= nan_seen;
+        uint32_t out[2];
+        pack_octet<BITS>(X, Z, out);
         if (eb < a.padded) {
-            const uint32_t keep = ok ? FULL : 0u;
             if (BITS == 8) {
-                uint2 o = make_uint2(word[0] & keep, word[(8 * BITS) / 32 > 1 ? 1 : 0] & keep);
-                *reinterpret_cast<uint2 *>(codes + eb) = o;
+                *reinterpret_cast<uint2 *>(codes + eb) = make_uint2(out[0], out[1]);
             } else if (BITS == 4) {
-                *reinterpret_cast<uint32_t *>(codes + (eb >> 1)) = word[0] & keep;
+                *reinterpret_cast<uint32_t *>(codes + (eb >> 1)) = out[0];
             } else {
-                *reinterpret_cast<uint16_t *>(codes + (eb >> 2)) = (uint16_t)(word[0] & keep);
+                *reinterpret_cast<uint16_t *>(codes + (eb >> 2)) = (uint16_t)out[0];
             }
         }
     }
@@ -433,7 +475,7 @@ cudaError_t launch_encode_v(const EncodeArgs &a, uint32_t K, cudaStream_t stream
     const uint64_t tiles = (a.padded + tile - 1) / tile;
     if (tiles == 0 || tiles * K > 0x7FFFFFFFull) return cudaErrorInvalidValue;
     dim3 grid((unsigned)(tiles * K), 1, 1), block(warps * 32u, 1, 1);
-    qesgd_encode_kernel<BITS, MODE, ANCHOR, VEC, V><<<grid, block, 0, stream>>>(a);
+    qesgd_encode_kernel<BITS, MODE, ANCHOR, VEC><<<grid, block, 0, stream>>>(a);
     return cudaGetLastError();
 }
 
