@@ -161,7 +161,7 @@ int qesgd_encode_batch(qesgd_ctx *ctx, const float *local, uint64_t local_stride
     const bool vec = aligned(local, 32) && aligned(anchor, 32) && (a.local_stride % 8 == 0);
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
-    const int e = qesgd_launch_encode(a, K, bits, scale_mode, vec, ctx->stream);
+    const int e = qesgd_launch_encode(a, K, bits, scale_mode, vec, ctx->sm_count, ctx->stream);
     if (e != 0) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return QESGD_OK;

@@ -15,6 +15,12 @@ namespace {
 
 constexpr uint32_t FULL = 0xFFFFFFFFu;
 constexpr int CHUNK = 256;  // elements covered by one warp-wide 256-bit load
+#ifndef QESGD_ENCODE_CHUNKS
+#define QESGD_ENCODE_CHUNKS 4  // chunks per warp in the encode kernel (2 or 4)
+#endif
+#ifndef QESGD_ENCODE_WARPS
+#define QESGD_ENCODE_WARPS 4   // warps per CTA unless a bucket needs more
+#endif
 
 // ---------------------------------------------------------------- memory ----
 __device__ __forceinline__ void ld256(const float *p, float (&v)[8])
@@ -156,14 +162,25 @@ struct MaxU32 {
     static __device__ __forceinline__ uint32_t op(uint32_t x, uint32_t y) { return max(x, y); }
 };
 
-// Reduces the four per-chunk partials of every lane over the lanes (and chunks) of a
+// Reduces the V per-chunk partials of every lane over the lanes (and chunks) of a
 // bucket, in the order of the balanced binary tree on element index: lanes xor 1, 2,
-// 4, (8), (16), then chunk pairs, then chunk quads.  The first two steps hand each
-// lane ONE chunk to carry on with (even/odd lanes split chunks {0,1}/{2,3}, then bit 1
-// of the lane splits the pair), so the rest of the tree costs one value per step
-// instead of four.  On return lane L holds the bucket total of chunk
-// 2*(L&1) + ((L>>1)&1) of its own lane group (for buckets >= 512 the chunks of one
-// bucket all hold its total).
+// 4, (8), (16), then chunk pairs, then chunk quads.  The first step(s) hand each lane
+// ONE chunk to carry on with (V = 4: even/odd lanes split chunks {0,1}/{2,3}, then
+// bit 1 of the lane splits the pair; V = 2: even lanes take chunk 0, odd lanes chunk
+// 1), so the rest of the tree costs one value per step instead of V.  On return lane
+// L holds the bucket total of chunk chunk_of_lane<V>(L) of its own lane group (once a
+// bucket spans several chunks, all of them hold its total).
+template <int V>
+__device__ __forceinline__ uint32_t chunk_of_lane(uint32_t lane)
+{
+    return V == 4 ? 2u * (lane & 1u) + ((lane >> 1) & 1u) : (lane & 1u);
+}
+template <int V>
+__device__ __forceinline__ uint32_t lane_of_chunk(uint32_t lane, int c)
+{
+    return V == 4 ? ((lane & 28u) | ((c >> 1) & 1) | ((c & 1) << 1)) : ((lane & 30u) | (c & 1));
+}
+
 template <typename R>
 __device__ __forceinline__ typename R::T reduce_chunks(const typename R::T (&t)[4], uint32_t lane,
                                                        uint32_t lb)
@@ -185,74 +202,68 @@ __device__ __forceinline__ typename R::T reduce_chunks(const typename R::T (&t)[
     return k;
 }
 
-// Buckets wider than a warp's 1024 elements: combine the totals of the wpb = bucket/1024
-// consecutive warps that share a bucket, adjacent pairs first.
 template <typename R>
-__device__ __forceinline__ typename R::T reduce_warps(typename R::T k, typename R::T *smem,
-                                                      uint32_t lane, uint32_t warp, uint32_t lb)
+__device__ __forceinline__ typename R::T reduce_chunks(const typename R::T (&t)[2], uint32_t lane,
+                                                       uint32_t lb)
 {
     typedef typename R::T T;
-    const uint32_t wpb = 1u << (lb - 10);
+    const bool b0 = lane & 1u;
+    T k = b0 ? t[1] : t[0];
+    const T s = b0 ? t[0] : t[1];
+    k = R::op(k, __shfl_xor_sync(FULL, s, 1));
+    k = R::op(k, __shfl_xor_sync(FULL, k, 2));
+    k = R::op(k, __shfl_xor_sync(FULL, k, 4));
+    if (lb >= 7) k = R::op(k, __shfl_xor_sync(FULL, k, 8));
+    if (lb >= 8) k = R::op(k, __shfl_xor_sync(FULL, k, 16));
+    if (lb >= 9) k = R::op(k, __shfl_xor_sync(FULL, k, 1));    // both chunks
+    return k;
+}
+
+// Buckets wider than a warp's V*256 elements: combine the totals of the wpb consecutive
+// warps that share a bucket (wpb a power of two <= 16), adjacent pairs first.
+template <typename R>
+__device__ __forceinline__ typename R::T reduce_warps(typename R::T k, typename R::T *smem,
+                                                      uint32_t lane, uint32_t warp, uint32_t wpb)
+{
+    typedef typename R::T T;
     if (lane == 0) smem[warp] = k;
     __syncthreads();
-    const uint32_t g0 = warp & ~(wpb - 1u);
-    T acc[8];
+    // lanes 0..wpb-1 (and every further group of wpb lanes) pick up the warps' totals; the
+    // xor butterfly over them is the balanced tree on warp order
+    T v = smem[(warp & ~(wpb - 1u)) + (lane & (wpb - 1u))];
 #pragma unroll
-    for (int i = 0; i < 8; ++i) acc[i] = smem[(g0 + i) & 7u];
-#pragma unroll
-    for (int w2 = 1; w2 < 8; w2 <<= 1) {
-        if ((uint32_t)w2 < wpb) {
-#pragma unroll
-            for (int i = 0; i < 8; i += 2 * w2) acc[i] = R::op(acc[i], acc[i + w2]);
-        }
-    }
-    return acc[0];
+    for (int off = 1; off < 16; off <<= 1)
+        if ((uint32_t)off < wpb) v = R::op(v, __shfl_xor_sync(FULL, v, off));
+    return v;
 }
 
 // ------------------------------------------------------------- encode -------
 // MODE: 0 = L2 norm, 1 = max magnitude, 2 = caller-given spacing.
-// A warp owns V = 4 chunks = 1024 consecutive elements, a CTA of 8 warps 8192.
+// A warp owns V chunks = V*256 consecutive elements, a CTA of W warps W*V*256.
 // Buckets are powers of two in [64, 8192]:
-//   bucket <= 256   : bucket/8 lanes of one chunk
-//   bucket <= 1024  : bucket/256 chunks of one warp
-//   bucket  > 1024  : bucket/1024 consecutive warps of the CTA (shared memory)
-template <int BITS, int MODE, bool ANCHOR, bool VEC>
-__global__ void __launch_bounds__(256) qesgd_encode_kernel(const EncodeArgs a)
+//   bucket <= 256     : bucket/8 lanes of one chunk
+//   bucket <= 256*V   : bucket/256 chunks of one warp
+//   bucket  > 256*V   : bucket/(256*V) consecutive warps of the CTA (shared memory)
+struct EncodeShared {
+    double part[2][16];     // cross-warp partial sums, double-buffered by iteration
+    uint32_t maxv[2][16];
+};
+
+// Everything after the deltas z of one warp tile are in registers: bucket scale,
+// Philox draws, stochastic rounding, packing, stores.  `iter` selects the half of the
+// cross-warp scratch (callers alternate it between consecutive tiles of one CTA).
+// FULL = the whole warp tile lies inside the vector: no store needs a bounds check.
+template <int BITS, int MODE, int V, bool FULL>
+__device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)[V][8],
+                                                 uint64_t warp_base, uint32_t k, uint32_t lane,
+                                                 uint32_t warp, EncodeShared &sh, uint32_t iter)
 {
-    constexpr int V = 4;
-    __shared__ double s_part[8];
-    __shared__ uint32_t s_max[8];
-
-    const uint32_t lane = threadIdx.x & 31u;
-    const uint32_t warp = threadIdx.x >> 5;
-    // Workers vary fastest over the grid: the K CTAs that share a tile of the anchor run
-    // close together in time, so the anchor comes from HBM once and from L2 K-1 times.
-    const uint32_t k = blockIdx.x % a.K;
-    const uint32_t tile = blockIdx.x / a.K;
+    constexpr uint32_t LOG2_WARP_ELEMS = V == 4 ? 10 : 9;
     const uint32_t lb = a.log2_bucket;
-    const float *__restrict__ local = a.local + (uint64_t)k * a.local_stride;
-    const uint64_t warp_base = ((uint64_t)tile * 8u + warp) * (uint64_t)(V * CHUNK);
-
-    // ---- loads: everything this lane needs is requested before any use -------
-    float z[V][8];
-#pragma unroll
-    for (int c = 0; c < V; ++c)
-        load_octet<VEC>(local, warp_base + (uint64_t)c * CHUNK + lane * 8u, a.d, z[c]);
-    if (ANCHOR) {
-        float w[V][8];
-#pragma unroll
-        for (int c = 0; c < V; ++c)
-            load_octet<VEC>(a.anchor, warp_base + (uint64_t)c * CHUNK + lane * 8u, a.d, w[c]);
-#pragma unroll
-        for (int c = 0; c < V; ++c)
-#pragma unroll
-            for (int j = 0; j < 8; ++j) z[c][j] = __fsub_rn(z[c][j], w[c][j]);
-    }
-
-    // ---- per-bucket scale: one value per lane, then handed back per chunk ------
     const float sf = (float)a.s;
     float my_scale, my_inv;
     bool flag = false;
+    // ---- per-bucket scale: one value per lane, then handed back per chunk ------
     if (MODE == 0) {
         // fp64 sum of squares over the balanced binary tree on index order.  The product
         // of two fp32 values is exact in fp64, so fma(z1,z1,z0*z0) is fl64(q0+q1).
@@ -268,7 +279,8 @@ __global__ void __launch_bounds__(256) qesgd_encode_kernel(const EncodeArgs a)
             t[c] = __dadd_rn(__dadd_rn(q[0], q[1]), __dadd_rn(q[2], q[3]));
         }
         double tot = reduce_chunks<SumF64>(t, lane, lb);
-        if (lb > 10) tot = reduce_warps<SumF64>(tot, s_part, lane, warp, lb);
+        if (lb > LOG2_WARP_ELEMS)
+            tot = reduce_warps<SumF64>(tot, sh.part[iter & 1u], lane, warp, 1u << (lb - LOG2_WARP_ELEMS));
         my_scale = __double2float_rn(__dsqrt_rn(tot));
     } else if (MODE == 1) {
         // Largest magnitude: bit patterns of |z| order like unsigned integers, and
@@ -281,7 +293,8 @@ __global__ void __launch_bounds__(256) qesgd_encode_kernel(const EncodeArgs a)
             for (int j = 0; j < 8; ++j) m[c] = max(m[c], __float_as_uint(z[c][j]) & 0x7FFFFFFFu);
         }
         uint32_t mm = reduce_chunks<MaxU32>(m, lane, lb);
-        if (lb > 10) mm = reduce_warps<MaxU32>(mm, s_max, lane, warp, lb);
+        if (lb > LOG2_WARP_ELEMS)
+            mm = reduce_warps<MaxU32>(mm, sh.maxv[iter & 1u], lane, warp, 1u << (lb - LOG2_WARP_ELEMS));
         my_scale = __uint_as_float(mm);
     } else {
         my_scale = a.fixed_scale;
@@ -304,12 +317,12 @@ __global__ void __launch_bounds__(256) qesgd_encode_kernel(const EncodeArgs a)
     for (int c = 0; c < V; ++c) {
         const uint64_t eb = warp_base + (uint64_t)c * CHUNK + lane * 8u;
         float scale = my_scale, inv = my_inv;
-        if (MODE != 2) {   // chunk c's bucket total sits in the lane of this quad with bits (c>>1, c&1)
-            const int src = (lane & 28u) | ((c >> 1) & 1) | ((c & 1) << 1);
+        if (MODE != 2) {   // fetch chunk c's bucket scale from the neighbour lane that carried it
+            const int src = (int)lane_of_chunk<V>(lane, c);
             scale = __shfl_sync(FULL, my_scale, src);
             inv = __shfl_sync(FULL, my_inv, src);
         }
-        if (eb < a.padded && ((uint32_t)eb & bucket_mask) == 0u) scales[eb >> lb] = scale;
+        if ((FULL || eb < a.padded) && ((uint32_t)eb & bucket_mask) == 0u) scales[eb >> lb] = scale;
 
         uint32_t x[4];
         const uint64_t blk = eb >> 3;
@@ -326,7 +339,7 @@ __global__ void __launch_bounds__(256) qesgd_encode_kernel(const EncodeArgs a)
         }
         uint32_t out[2];
         pack_octet<BITS>(X, Z, out);
-        if (eb < a.padded) {
+        if (FULL || eb < a.padded) {
             if (BITS == 8) {
                 *reinterpret_cast<uint2 *>(codes + eb) = make_uint2(out[0], out[1]);
             } else if (BITS == 4) {
@@ -337,6 +350,56 @@ __global__ void __launch_bounds__(256) qesgd_encode_kernel(const EncodeArgs a)
         }
     }
     if (flag) atomicOr(a.status, QESGD_STATUS_NONFINITE);
+}
+
+// One CTA per (tile, worker); every lane requests all of its 256-bit loads before it
+// uses any of them, and several CTAs per SM overlap one another's load and arithmetic
+// phases.  VEC = false (pointers not 32-byte aligned) falls back to scalar loads.
+template <int BITS, int MODE, bool ANCHOR, bool VEC, int V, int WARPS>
+__global__ void __launch_bounds__(WARPS * 32, 1024 / (WARPS * 32))
+    qesgd_encode_kernel(const EncodeArgs a)
+{
+    __shared__ EncodeShared sh;
+    const uint32_t lane = threadIdx.x & 31u;
+    const uint32_t warp = threadIdx.x >> 5;
+    // Workers vary fastest over the grid: the K CTAs that share a tile of the anchor run
+    // close together in time, so the anchor comes from HBM once and from L2 K-1 times.
+    const uint32_t k = blockIdx.x % a.K;
+    const uint32_t tile = blockIdx.x / a.K;
+    const float *__restrict__ local = a.local + (uint64_t)k * a.local_stride;
+    const uint64_t warp_base = ((uint64_t)tile * WARPS + warp) * (uint64_t)(V * CHUNK);
+
+    float z[V][8];
+    if (VEC && warp_base + V * CHUNK <= a.d) {   // the whole warp tile is inside the vector
+        const float *__restrict__ p = local + warp_base + lane * 8u;
+#pragma unroll
+        for (int c = 0; c < V; ++c) ld256(p + c * CHUNK, z[c]);
+        if (ANCHOR) {
+            const float *__restrict__ q = a.anchor + warp_base + lane * 8u;
+            float w[V][8];
+#pragma unroll
+            for (int c = 0; c < V; ++c) ld256(q + c * CHUNK, w[c]);
+#pragma unroll
+            for (int c = 0; c < V; ++c)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) z[c][j] = __fsub_rn(z[c][j], w[c][j]);
+        }
+        encode_warp_tile<BITS, MODE, V, true>(a, z, warp_base, k, lane, warp, sh, 0u);
+        return;
+    }
+#pragma unroll
+    for (int c = 0; c < V; ++c)
+        load_octet<VEC>(local, warp_base + (uint64_t)c * CHUNK + lane * 8u, a.d, z[c]);
+    if (ANCHOR) {
+#pragma unroll
+        for (int c = 0; c < V; ++c) {
+            float w[8];
+            load_octet<VEC>(a.anchor, warp_base + (uint64_t)c * CHUNK + lane * 8u, a.d, w);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) z[c][j] = __fsub_rn(z[c][j], w[j]);
+        }
+    }
+    encode_warp_tile<BITS, MODE, V, false>(a, z, warp_base, k, lane, warp, sh, 0u);
 }
 
 // ------------------------------------------------------------- decode -------
@@ -465,50 +528,62 @@ __global__ void __launch_bounds__(256) qesgd_decode_average_apply_kernel(const D
 }
 
 // ------------------------------------------------------------ dispatch ------
-template <int BITS, int MODE, bool ANCHOR, bool VEC>
-cudaError_t launch_encode_v(const EncodeArgs &a, uint32_t K, cudaStream_t stream)
+template <int BITS, int MODE, bool ANCHOR, bool VEC, int WARPS>
+cudaError_t launch_encode_w(const EncodeArgs &a, uint32_t K, cudaStream_t stream)
 {
-    constexpr int V = 4;
-    constexpr uint32_t warps = 8;  // 8 warps * V * 256 = 8192 elements: the largest bucket fits
-    static_assert(warps * V * CHUNK >= QESGD_MAX_BUCKET, "a bucket never leaves its CTA");
-    const uint64_t tile = (uint64_t)warps * V * CHUNK;
+    constexpr int V = QESGD_ENCODE_CHUNKS;
+    const uint64_t tile = (uint64_t)WARPS * V * CHUNK;
     const uint64_t tiles = (a.padded + tile - 1) / tile;
     if (tiles == 0 || tiles * K > 0x7FFFFFFFull) return cudaErrorInvalidValue;
-    dim3 grid((unsigned)(tiles * K), 1, 1), block(warps * 32u, 1, 1);
-    qesgd_encode_kernel<BITS, MODE, ANCHOR, VEC><<<grid, block, 0, stream>>>(a);
+    dim3 grid((unsigned)(tiles * K), 1, 1), block(WARPS * 32u, 1, 1);
+    qesgd_encode_kernel<BITS, MODE, ANCHOR, VEC, V, WARPS><<<grid, block, 0, stream>>>(a);
     return cudaGetLastError();
 }
 
+template <int BITS, int MODE, bool ANCHOR, bool VEC>
+cudaError_t launch_encode_v(const EncodeArgs &a, uint32_t K, int sm_count, cudaStream_t stream)
+{
+    (void)sm_count;
+    constexpr int V = QESGD_ENCODE_CHUNKS;
+    constexpr uint32_t SMALL = QESGD_ENCODE_WARPS;        // warps of the usual CTA
+    constexpr uint32_t LARGE = QESGD_MAX_BUCKET / (V * CHUNK);   // enough for the widest bucket
+    // a bucket never leaves its CTA
+    if ((1u << a.log2_bucket) <= SMALL * V * CHUNK)
+        return launch_encode_w<BITS, MODE, ANCHOR, VEC, SMALL>(a, K, stream);
+    return launch_encode_w<BITS, MODE, ANCHOR, VEC, (LARGE > SMALL ? LARGE : SMALL)>(a, K, stream);
+}
+
 template <int BITS, int MODE>
-cudaError_t launch_encode_m(const EncodeArgs &a, uint32_t K, bool vec, cudaStream_t stream)
+cudaError_t launch_encode_m(const EncodeArgs &a, uint32_t K, bool vec, int sm_count,
+                            cudaStream_t stream)
 {
     if (a.anchor)
-        return vec ? launch_encode_v<BITS, MODE, true, true>(a, K, stream)
-                   : launch_encode_v<BITS, MODE, true, false>(a, K, stream);
-    return vec ? launch_encode_v<BITS, MODE, false, true>(a, K, stream)
-               : launch_encode_v<BITS, MODE, false, false>(a, K, stream);
+        return vec ? launch_encode_v<BITS, MODE, true, true>(a, K, sm_count, stream)
+                   : launch_encode_v<BITS, MODE, true, false>(a, K, sm_count, stream);
+    return vec ? launch_encode_v<BITS, MODE, false, true>(a, K, sm_count, stream)
+               : launch_encode_v<BITS, MODE, false, false>(a, K, sm_count, stream);
 }
 
 template <int BITS>
 cudaError_t launch_encode_b(const EncodeArgs &a, uint32_t K, uint32_t mode, bool vec,
-                            cudaStream_t stream)
+                            int sm_count, cudaStream_t stream)
 {
     switch (mode) {
-        case QESGD_SCALE_NORM: return launch_encode_m<BITS, 0>(a, K, vec, stream);
-        case QESGD_SCALE_MAX: return launch_encode_m<BITS, 1>(a, K, vec, stream);
-        default: return launch_encode_m<BITS, 2>(a, K, vec, stream);
+        case QESGD_SCALE_NORM: return launch_encode_m<BITS, 0>(a, K, vec, sm_count, stream);
+        case QESGD_SCALE_MAX: return launch_encode_m<BITS, 1>(a, K, vec, sm_count, stream);
+        default: return launch_encode_m<BITS, 2>(a, K, vec, sm_count, stream);
     }
 }
 
 }  // namespace
 
 int qesgd_launch_encode(const EncodeArgs &a, uint32_t K, uint32_t bits, uint32_t scale_mode,
-                        bool vec, cudaStream_t stream)
+                        bool vec, int sm_count, cudaStream_t stream)
 {
     switch (bits) {
-        case 2: return (int)launch_encode_b<2>(a, K, scale_mode, vec, stream);
-        case 4: return (int)launch_encode_b<4>(a, K, scale_mode, vec, stream);
-        default: return (int)launch_encode_b<8>(a, K, scale_mode, vec, stream);
+        case 2: return (int)launch_encode_b<2>(a, K, scale_mode, vec, sm_count, stream);
+        case 4: return (int)launch_encode_b<4>(a, K, scale_mode, vec, sm_count, stream);
+        default: return (int)launch_encode_b<8>(a, K, scale_mode, vec, sm_count, stream);
     }
 }
 

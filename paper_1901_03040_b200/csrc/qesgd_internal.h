@@ -55,7 +55,7 @@ struct DecodeArgs {
 
 // Launchers (defined in qesgd_codec.cu / qesgd_lr.cu).  Return a cudaError_t as int.
 int qesgd_launch_encode(const EncodeArgs &a, uint32_t K, uint32_t bits, uint32_t scale_mode,
-                        bool vec, cudaStream_t stream);
+                        bool vec, int sm_count, cudaStream_t stream);
 int qesgd_launch_decode(const DecodeArgs &a, uint32_t bits, bool vec, cudaStream_t stream);
 int qesgd_launch_decode_average_apply(const DecodeArgs &a, uint32_t bits, bool vec,
                                       cudaStream_t stream);
