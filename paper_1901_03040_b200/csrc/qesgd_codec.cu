@@ -415,17 +415,6 @@ __device__ __forceinline__ float code_value(uint32_t word, int slot, float step)
     return __uint_as_float(__float_as_uint(__fmul_rn(lf, step)) ^ sign31);
 }
 
-// acc += +-level * step with one rounding (the sign is folded into the multiplier).
-template <int BITS>
-__device__ __forceinline__ void accumulate_code(uint32_t word, int slot, float step, float &acc)
-{
-    constexpr uint32_t LEVEL_MASK = (1u << (BITS - 1)) - 1u;
-    const uint32_t lv = (word >> (slot * BITS)) & LEVEL_MASK;
-    const float lf = __fsub_rn(__uint_as_float(0x4B000000u | lv), 8388608.0f);
-    const uint32_t sign31 = (word << (31 - (slot * BITS + BITS - 1))) & 0x80000000u;
-    acc = __fmaf_rn(lf, __uint_as_float(__float_as_uint(step) ^ sign31), acc);
-}
-
 // The packed codes of the octet starting at element eb: 8*BITS bits.
 template <int BITS>
 __device__ __forceinline__ void load_codes(const uint8_t *__restrict__ codes, uint64_t eb,
@@ -467,12 +456,45 @@ __global__ void __launch_bounds__(256) qesgd_decode_kernel(const DecodeArgs a)
 }
 
 // -------------------------------------------- decode + average + apply ------
+// acc[j] += +-level_j * step for the 8 codes of one octet (one rounding each: the sign
+// is folded into the multiplier).  Levels are spliced into the mantissa of 2^23.
+template <int BITS>
+__device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], float step, float (&acc)[8])
+{
+    const uint32_t sb = __float_as_uint(step);
+    if (BITS == 8) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const uint32_t lv = cw[h] & 0x7F7F7F7Fu;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                // byte j of lv under the upper three bytes of 2^23
+                const float m = __uint_as_float(__byte_perm(lv, 0x4B000000u, 0x7650 + j));
+                const uint32_t sign31 = (j == 3 ? cw[h] : (cw[h] << (24 - 8 * j))) & 0x80000000u;
+                acc[4 * h + j] = __fmaf_rn(__fsub_rn(m, 8388608.0f), __uint_as_float(sb ^ sign31),
+                                           acc[4 * h + j]);
+            }
+        }
+    } else {
+        constexpr uint32_t LEVEL_MASK = (1u << (BITS - 1)) - 1u;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t m = ((cw[0] >> (j * BITS)) & LEVEL_MASK) | 0x4B000000u;
+            const uint32_t sign31 = (cw[0] << (31 - (j * BITS + BITS - 1))) & 0x80000000u;
+            acc[j] = __fmaf_rn(__fsub_rn(__uint_as_float(m), 8388608.0f),
+                               __uint_as_float(sb ^ sign31), acc[j]);
+        }
+    }
+}
+
 // One octet per lane, one chunk of 256 elements per warp.  The K grid spacings
 // fl32(scale/s) a chunk needs are computed once per warp (one division per lane)
-// and handed out by shuffle, so the inner loop per code is shift/mask/fma work.
+// and handed out by shuffle; code words are fetched eight workers at a time so that
+// eight independent loads are in flight per lane before the first is used.
 template <int BITS, bool VEC>
 __global__ void __launch_bounds__(256) qesgd_decode_average_apply_kernel(const DecodeArgs a)
 {
+    constexpr int BATCH = 8;
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp_eb =
         (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * (uint64_t)CHUNK;
@@ -484,10 +506,10 @@ __global__ void __launch_bounds__(256) qesgd_decode_average_apply_kernel(const D
     const uint64_t bucket0 = warp_eb >> lb;
     const uint32_t per_pass = 32u / nbw;                        // workers per pass
     const float sf = (float)a.s;
-    const bool live = eb < a.d;
+    const bool vec_ok = VEC && eb + 8 <= a.d;
 
     float w[8];
-    if (VEC && eb + 8 <= a.d) {
+    if (vec_ok) {
         ld256_rw(a.param + eb, w);
     } else {
 #pragma unroll
@@ -497,8 +519,12 @@ __global__ void __launch_bounds__(256) qesgd_decode_average_apply_kernel(const D
 #pragma unroll
     for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
 
-    const uint8_t *__restrict__ codes = reinterpret_cast<const uint8_t *>(a.codes);
-    constexpr int PER_WORD = 32 / BITS;
+    // Lanes past the padded length of the streams read the warp's first octet instead
+    // (their result is never stored), so no load needs a predicate.
+    const uint64_t safe_eb = eb < (a.nb << lb) ? eb : warp_eb;
+    const uint8_t *__restrict__ cp =
+        reinterpret_cast<const uint8_t *>(a.codes) + (safe_eb >> 3) * (uint64_t)BITS;
+
     for (uint32_t k0 = 0; k0 < a.K; k0 += per_pass) {
         const uint32_t kk = k0 + lane / nbw;
         const uint64_t bb = bucket0 + (lane % nbw);
@@ -506,19 +532,37 @@ __global__ void __launch_bounds__(256) qesgd_decode_average_apply_kernel(const D
         if (kk < a.K && bb < a.nb)
             st = __fdiv_rn(__ldg(a.scales + (uint64_t)kk * a.scale_stride + bb), sf);
         const uint32_t count = min(per_pass, a.K - k0);
-#pragma unroll 4
-        for (uint32_t i = 0; i < count; ++i) {
-            const float step = __shfl_sync(FULL, st, i * nbw + sub);
-            uint32_t cw[2] = {0u, 0u};
-            if (live) load_codes<BITS>(codes + (uint64_t)(k0 + i) * a.code_stride, eb, cw);
+        for (uint32_t i0 = 0; i0 < count; i0 += BATCH) {
+            uint32_t cw[BATCH][2];
 #pragma unroll
-            for (int j = 0; j < 8; ++j) accumulate_code<BITS>(cw[j / PER_WORD], j % PER_WORD, step, acc[j]);
+            for (int i = 0; i < BATCH; ++i) {
+                cw[i][0] = cw[i][1] = 0u;
+                if (i0 + i < count) {
+                    const uint8_t *q = cp + (uint64_t)(k0 + i0 + i) * a.code_stride;
+                    if (BITS == 8) {
+                        const uint2 v = __ldg(reinterpret_cast<const uint2 *>(q));
+                        cw[i][0] = v.x;
+                        cw[i][1] = v.y;
+                    } else if (BITS == 4) {
+                        cw[i][0] = __ldg(reinterpret_cast<const uint32_t *>(q));
+                    } else {
+                        cw[i][0] = __ldg(reinterpret_cast<const uint16_t *>(q));
+                    }
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < BATCH; ++i) {
+                if (i0 + i < count) {   // uniform across the warp
+                    const float step = __shfl_sync(FULL, st, (i0 + i) * nbw + sub);
+                    accumulate_octet<BITS>(cw[i], step, acc);
+                }
+            }
         }
     }
     const float inv_k = __fdiv_rn(1.0f, (float)a.K);
 #pragma unroll
     for (int j = 0; j < 8; ++j) w[j] = __fmaf_rn(acc[j], inv_k, w[j]);
-    if (VEC && eb + 8 <= a.d) {
+    if (vec_ok) {
         st256(a.param + eb, w);
     } else {
 #pragma unroll
