@@ -456,12 +456,54 @@ __global__ void __launch_bounds__(256) qesgd_decode_kernel(const DecodeArgs a)
 }
 
 // -------------------------------------------- decode + average + apply ------
-// acc[j] += +-level_j * step for the 8 codes of one octet (one rounding each: the sign
-// is folded into the multiplier).  Levels are spliced into the mantissa of 2^23.
+// Packed fp32 pairs (sm_100: add/fma on two floats per instruction).
+__device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi)
+{
+    uint64_t p;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p) : "r"(lo), "r"(hi));
+    return p;
+}
+__device__ __forceinline__ void unpack2(uint64_t p, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+// (a & b) | c and (a & b) ^ c as one three-input logic operation each
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t and_xor(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+// acc += +-level * step for the 8 codes of one octet, two elements per arithmetic
+// instruction (acc[p] holds elements 2p, 2p+1).  One rounding per product-sum: the sign
+// is folded into the multiplier.  Levels are spliced into the mantissa of 2^23 and the
+// 2^23 is subtracted again, which converts them to float exactly.
 template <int BITS>
-__device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], float step, float (&acc)[8])
+__device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], float step,
+                                                 uint64_t (&acc)[4])
 {
     const uint32_t sb = __float_as_uint(step);
+    const uint64_t neg_magic = pack2(0xCB000000u, 0xCB000000u);   // (-2^23, -2^23)
+    uint32_t m[8], sg[8];
     if (BITS == 8) {
 #pragma unroll
         for (int h = 0; h < 2; ++h) {
@@ -469,22 +511,22 @@ __device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], float 
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 // byte j of lv under the upper three bytes of 2^23
-                const float m = __uint_as_float(__byte_perm(lv, 0x4B000000u, 0x7650 + j));
-                const uint32_t sign31 = (j == 3 ? cw[h] : (cw[h] << (24 - 8 * j))) & 0x80000000u;
-                acc[4 * h + j] = __fmaf_rn(__fsub_rn(m, 8388608.0f), __uint_as_float(sb ^ sign31),
-                                           acc[4 * h + j]);
+                m[4 * h + j] = __byte_perm(lv, 0x4B000000u, 0x7650 + j);
+                sg[4 * h + j] = and_xor(j == 3 ? cw[h] : (cw[h] << (24 - 8 * j)), 0x80000000u, sb);
             }
         }
     } else {
         constexpr uint32_t LEVEL_MASK = (1u << (BITS - 1)) - 1u;
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const uint32_t m = ((cw[0] >> (j * BITS)) & LEVEL_MASK) | 0x4B000000u;
-            const uint32_t sign31 = (cw[0] << (31 - (j * BITS + BITS - 1))) & 0x80000000u;
-            acc[j] = __fmaf_rn(__fsub_rn(__uint_as_float(m), 8388608.0f),
-                               __uint_as_float(sb ^ sign31), acc[j]);
+            m[j] = and_or(cw[0] >> (j * BITS), LEVEL_MASK, 0x4B000000u);
+            sg[j] = and_xor(cw[0] << (31 - (j * BITS + BITS - 1)), 0x80000000u, sb);
         }
     }
+#pragma unroll
+    for (int p = 0; p < 4; ++p)
+        acc[p] = fma2(add2(pack2(m[2 * p], m[2 * p + 1]), neg_magic),
+                      pack2(sg[2 * p], sg[2 * p + 1]), acc[p]);
 }
 
 // One octet per lane, one chunk of 256 elements per warp.  The K grid spacings
@@ -515,9 +557,7 @@ __global__ void __launch_bounds__(256) qesgd_decode_average_apply_kernel(const D
 #pragma unroll
         for (int j = 0; j < 8; ++j) w[j] = (eb + j < a.d) ? a.param[eb + j] : 0.0f;
     }
-    float acc[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j) acc[j] = 0.0f;
+    uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};   // four pairs of +0.0f
 
     // Lanes past the padded length of the streams read the warp's first octet instead
     // (their result is never stored), so no load needs a predicate.
@@ -561,7 +601,12 @@ __global__ void __launch_bounds__(256) qesgd_decode_average_apply_kernel(const D
     }
     const float inv_k = __fdiv_rn(1.0f, (float)a.K);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) w[j] = __fmaf_rn(acc[j], inv_k, w[j]);
+    for (int p = 0; p < 4; ++p) {
+        float lo, hi;
+        unpack2(acc[p], lo, hi);
+        w[2 * p] = __fmaf_rn(lo, inv_k, w[2 * p]);
+        w[2 * p + 1] = __fmaf_rn(hi, inv_k, w[2 * p + 1]);
+    }
     if (vec_ok) {
         st256(a.param + eb, w);
     } else {
