@@ -51,6 +51,7 @@ extern "C" {
 #define QESGD_EINVAL (-1) /* NULL / misaligned pointer, unsupported bits, bucket, s, K, mode */
 #define QESGD_ECUDA (-2)  /* CUDA runtime or launch error; see qesgd_last_cuda_error      */
 #define QESGD_ENOMEM (-3) /* host or device allocation failed (qesgd_create only)          */
+#define QESGD_ELIMIT (-4) /* size beyond the fixed scratch of a no-allocation entry point   */
 
 #define QESGD_SCALE_NORM 0u  /* scale = L2 norm of the bucket's delta              */
 #define QESGD_SCALE_MAX 1u   /* scale = largest magnitude of the bucket's delta    */
@@ -63,6 +64,7 @@ extern "C" {
 #define QESGD_MIN_BUCKET 64u
 #define QESGD_MAX_BUCKET 8192u
 #define QESGD_MAX_LR_BATCH 1024u
+#define QESGD_NOALLOC_MAX_LR_BATCH 256u /* rows per step of qesgd_lr_sgd_step_noalloc */
 
 typedef struct qesgd_ctx qesgd_ctx;
 
@@ -151,6 +153,32 @@ int qesgd_lr_local_epoch(qesgd_ctx *ctx, const float *X, const float *y, uint64_
 int qesgd_lr_local_epoch_batch(qesgd_ctx *ctx, const float *X, const float *y, uint64_t n_local,
                                uint64_t d, uint32_t K, uint32_t batch, float lr, float *u,
                                uint64_t u_stride);
+
+/*
+ * The paper has no counterpart for this entry point; it exists for callers that are
+ * not allowed to allocate device memory at the moment they need a step: code running
+ * inside a memory-pool or allocator callback, a real-time loop that must not touch
+ * the driver's allocator, or a host that was handed a fixed memory budget and may
+ * not create a qesgd_ctx (qesgd_create allocates).  It is qesgd_lr_sgd_step without
+ * a context: same kernels, same arithmetic, same result.
+ *
+ * The partial margins the two passes exchange live in a fixed array inside the
+ * library image (64 KB of device memory on every GPU that loads the library, held
+ * until the process exits) instead of a context's workspace.  Consequences:
+ *   - m must not exceed QESGD_NOALLOC_MAX_LR_BATCH; larger batches return
+ *     QESGD_ELIMIT and enqueue nothing.  d is unlimited.
+ *   - the call works on the CURRENT device and enqueues on cuda_stream (NULL = legacy
+ *     default stream); Xb, yb, u are device pointers as for qesgd_lr_sgd_step.
+ *   - it calls no cudaMalloc / cudaFree and nothing that allocates.  The first call
+ *     on each device looks up the array's device address (a query, not an
+ *     allocation); make that first call before starting any stream capture.
+ *   - every call shares the one array, which keeps the previous call's contents.
+ *     Nothing in it has to start at zero: the first pass overwrites every slot the
+ *     second pass reads.  Two calls that overlap on the GPU (different streams, or
+ *     different host threads) race on it: serialise them on one stream.
+ */
+int qesgd_lr_sgd_step_noalloc(void *cuda_stream, const float *Xb, const float *yb, uint32_t m,
+                              uint64_t d, float lr, float *u);
 
 /* Waits for the stream, copies the status word to *flags_out (host) and clears it. */
 int qesgd_status(qesgd_ctx *ctx, uint32_t *flags_out);

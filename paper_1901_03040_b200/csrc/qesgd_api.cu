@@ -301,6 +301,7 @@ const char *qesgd_strerror(int code)
         case QESGD_EINVAL: return "invalid argument";
         case QESGD_ECUDA: return "CUDA error (see qesgd_last_cuda_error)";
         case QESGD_ENOMEM: return "out of memory";
+        case QESGD_ELIMIT: return "size exceeds the fixed scratch of the no-allocation entry point";
         default: return "unknown error";
     }
 }

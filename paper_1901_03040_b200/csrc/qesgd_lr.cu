@@ -9,6 +9,8 @@
 //           (lr/m) * y_j / (1 + exp(y_j m_j)) in shared memory and updates 512 columns
 //           of u with sum_j coef_j x_jc.  X_B is normally still in L2 for this pass.
 // No tensor cores: with m = 64 rows the work is 64 dot products, bound by memory.
+#include <mutex>
+
 #include "qesgd_internal.h"
 
 namespace {
@@ -175,4 +177,54 @@ int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float 
     e = cudaGetLastError();
     if (e == cudaSuccess) *launched = 2;
     return (int)e;
+}
+
+// ---------------------------------------------------------------------------
+// Entry point that allocates nothing: the partial margins go to a fixed array in
+// the library image.  In host code the array's name is only a handle; the device
+// address is looked up once per device with cudaGetSymbolAddress and cached.
+// ---------------------------------------------------------------------------
+namespace {
+
+constexpr uint32_t NOALLOC_FLOATS = MAX_PARTS * QESGD_NOALLOC_MAX_LR_BATCH;   // 64 KB
+static __device__ __align__(256) float g_noalloc_lr_scratch[NOALLOC_FLOATS];
+
+constexpr int MAX_DEVICES = 64;
+std::mutex g_noalloc_mutex;
+float *g_noalloc_ptr[MAX_DEVICES] = {nullptr};
+
+// Device address of the scratch array on the current device; looked up on first use.
+cudaError_t noalloc_scratch(float **out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_noalloc_lr_scratch);
+        if (e != cudaSuccess) return e;
+        g_noalloc_ptr[dev] = static_cast<float *>(p);
+    }
+    *out = g_noalloc_ptr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int qesgd_lr_sgd_step_noalloc(void *cuda_stream, const float *Xb, const float *yb,
+                                         uint32_t m, uint64_t d, float lr, float *u)
+{
+    if (m < 1) return QESGD_EINVAL;
+    if (m > QESGD_NOALLOC_MAX_LR_BATCH) return QESGD_ELIMIT;
+    if (d == 0) return QESGD_OK;
+    if (!Xb || !yb || !u) return QESGD_EINVAL;
+    if (((uintptr_t)Xb | (uintptr_t)yb | (uintptr_t)u) % 4 != 0) return QESGD_EINVAL;
+    float *scratch = nullptr;
+    if (noalloc_scratch(&scratch) != cudaSuccess) return QESGD_ECUDA;
+    int launched = 0;
+    const int e = qesgd_launch_lr_step(Xb, 0, yb, 0, m, d, 1, lr, u, 0, scratch, NOALLOC_FLOATS,
+                                       (cudaStream_t)cuda_stream, &launched);
+    return e == 0 ? QESGD_OK : QESGD_ECUDA;
 }

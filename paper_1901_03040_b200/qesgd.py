@@ -12,8 +12,9 @@ LIB_PATH = os.path.join(_HERE, "libqesgd.so")
 
 SCALE_NORM, SCALE_MAX, SCALE_FIXED = 0, 1, 2
 STATUS_NONFINITE = 1
-OK, EINVAL, ECUDA, ENOMEM = 0, -1, -2, -3
+OK, EINVAL, ECUDA, ENOMEM, ELIMIT = 0, -1, -2, -3, -4
 MAX_WORKERS, MIN_BUCKET, MAX_BUCKET, MAX_LR_BATCH = 64, 64, 8192, 1024
+NOALLOC_MAX_LR_BATCH = 256
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(
@@ -40,6 +41,7 @@ SIGNATURES = {
     "qesgd_lr_sgd_step": (_int, [_vp, _vp, _vp, _u32, _u64, _f32, _vp]),
     "qesgd_lr_local_epoch": (_int, [_vp, _vp, _vp, _u64, _u64, _u32, _f32, _vp]),
     "qesgd_lr_local_epoch_batch": (_int, [_vp, _vp, _vp, _u64, _u64, _u32, _u32, _f32, _vp, _u64]),
+    "qesgd_lr_sgd_step_noalloc": (_int, [_vp, _vp, _vp, _u32, _u64, _f32, _vp]),
     "qesgd_status": (_int, [_vp, C.POINTER(_u32)]),
     "qesgd_launch_count": (_u64, [_vp]),
     "qesgd_last_cuda_error": (_int, [_vp]),
@@ -151,6 +153,17 @@ class Context:
 
     def qesgd_launch_count(self):
         return int(lib.qesgd_launch_count(self._h))
+
+
+def qesgd_lr_sgd_step_noalloc(stream, Xb, yb, m, d, lr, u):
+    """One logistic SGD step on the current device without a context and without any
+    allocation by the library: for callers that must not allocate device memory when
+    they take the step (the scratch is a fixed 64 KB array inside the library; at most
+    NOALLOC_MAX_LR_BATCH rows; calls must not overlap on the GPU)."""
+    rc = lib.qesgd_lr_sgd_step_noalloc(C.c_void_p(stream.cuda_stream if stream is not None else 0),
+                                       _ptr(Xb), _ptr(yb), m, d, lr, _ptr(u))
+    if rc != OK:
+        raise QesgdError(rc)
 
 
 def alloc_stream_buffers(K, d, bucket, bits, device):
