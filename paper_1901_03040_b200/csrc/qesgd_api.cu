@@ -148,8 +148,10 @@ int qesgd_encode_batch(qesgd_ctx *ctx, const float *local, uint64_t local_stride
     a.log2_bucket = (uint32_t)log2_exact(bucket);
     a.s = s;
     a.fixed_scale = scale_mode == QESGD_SCALE_FIXED ? (float)s * fixed_delta : 0.0f;
-    a.key0 = (uint32_t)seed;
-    a.key1 = (uint32_t)(seed >> 32);
+    for (uint32_t r = 0; r < 10; ++r) {   // Philox4x32 key schedule (Weyl sequence)
+        a.round_key[r][0] = (uint32_t)seed + r * 0x9E3779B9u;
+        a.round_key[r][1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
+    }
     a.worker0 = worker0;
     a.epoch = epoch;
     a.K = K;

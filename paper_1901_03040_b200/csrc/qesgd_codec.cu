@@ -18,6 +18,9 @@ constexpr int CHUNK = 256;  // elements covered by one warp-wide 256-bit load
 #ifndef QESGD_ENCODE_CHUNKS
 #define QESGD_ENCODE_CHUNKS 4  // chunks per warp in the encode kernel (2 or 4)
 #endif
+#ifndef QESGD_ENCODE_MIN_WARPS
+#define QESGD_ENCODE_MIN_WARPS 24  // resident warps per SM the register budget is set for
+#endif
 #ifndef QESGD_ENCODE_WARPS
 #define QESGD_ENCODE_WARPS 4   // warps per CTA unless a bucket needs more
 #endif
@@ -66,20 +69,20 @@ __device__ __forceinline__ void load_octet(const float *__restrict__ p, uint64_t
 // published round function: two 32x32->64 multiplies, the high halves xor'ed with
 // the other counter words and the round key; the key grows by the Weyl constants.
 __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                              uint32_t k0, uint32_t k1, uint32_t (&x)[4])
+                                              const uint32_t (&rk)[10][2], uint32_t (&x)[4])
 {
+    // rk[r] = key + r * (0x9E3779B9, 0xBB67AE85): the ten round keys, prepared on the host so
+    // that they reach the xor as kernel-parameter operands instead of per-thread additions
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
         const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
         const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
-        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
-        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk[r][0];
+        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk[r][1];
         c1 = (uint32_t)p1;
         c3 = (uint32_t)p0;
         c0 = n0;
         c2 = n2;
-        k0 += 0x9E3779B9u;
-        k1 += 0xBB67AE85u;
     }
     x[0] = c0; x[1] = c1; x[2] = c2; x[3] = c3;
 }
@@ -326,7 +329,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
 
         uint32_t x[4];
         const uint64_t blk = eb >> 3;
-        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.worker0 + k, a.epoch, a.key0, a.key1, x);
+        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.worker0 + k, a.epoch, a.round_key, x);
 
         uint32_t X[8], Z[8];
 #pragma unroll
@@ -356,7 +359,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
 // uses any of them, and several CTAs per SM overlap one another's load and arithmetic
 // phases.  VEC = false (pointers not 32-byte aligned) falls back to scalar loads.
 template <int BITS, int MODE, bool ANCHOR, bool VEC, int V, int WARPS>
-__global__ void __launch_bounds__(WARPS * 32, 1024 / (WARPS * 32))
+__global__ void __launch_bounds__(WARPS * 32, QESGD_ENCODE_MIN_WARPS / WARPS)
     qesgd_encode_kernel(const EncodeArgs a)
 {
     __shared__ EncodeShared sh;

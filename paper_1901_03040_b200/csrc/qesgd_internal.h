@@ -30,7 +30,7 @@ struct EncodeArgs {
     uint32_t log2_bucket;
     uint32_t s;
     float fixed_scale;      // fl32(s * delta), FIXED mode only
-    uint32_t key0, key1;    // seed low / high
+    uint32_t round_key[10][2];  // Philox round keys: seed + r * Weyl constants
     uint32_t worker0, epoch;
     uint32_t K;             // workers in this launch
     uint32_t *codes;
