@@ -22,7 +22,7 @@ constexpr int CHUNK = 256;  // elements covered by one warp-wide 256-bit load
 #define QESGD_ENCODE_MIN_WARPS 24  // resident warps per SM the register budget is set for
 #endif
 #ifndef QESGD_ENCODE_WARPS
-#define QESGD_ENCODE_WARPS 4   // warps per CTA unless a bucket needs more
+#define QESGD_ENCODE_WARPS 1   // warps per CTA unless a bucket needs more
 #endif
 
 // ---------------------------------------------------------------- memory ----
