@@ -300,15 +300,24 @@ def run_ours(args):
 
 
 def load_traffic(kernel, workload):
-    """DRAM bytes per launch from the committed ncu summary, if one matches this kernel build."""
-    path = os.path.join(ROOT, "profiles", "traffic.json")
-    if not os.path.exists(path):
-        return None
+    """DRAM bytes (read + write) per launch from the committed ncu summary; None when there is
+    no capture for this kernel and workload, or the kernel source has changed since."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "dram_traffic_bench_c4.txt")
+    src = os.path.join(ROOT, "paper_1901_03040_b200", "csrc", "qesgd_codec.cu")
     try:
+        with open(src, "rb") as fh:
+            sha = hashlib.sha256(fh.read()).hexdigest()
+        value, sha_ok = None, False
         with open(path) as fh:
-            table = json.load(fh)
-        return table.get(f"{kernel}:{workload}")
-    except (OSError, ValueError):
+            for line in fh:
+                f = line.split()
+                if len(f) >= 2 and f[0] == "source_sha256":
+                    sha_ok = f[1] == sha
+                elif f and f[0] == f"{kernel}:{workload}" and "total_bytes" in f:
+                    value = float(f[f.index("total_bytes") + 1])
+        return value if sha_ok else None
+    except OSError:
         return None
 
 
@@ -534,7 +543,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=["c4", "c3", "c5", "c2", "c1"], default="c4")
@@ -542,7 +551,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-sample-elems", type=int, default=12_778_496)
-    ap.add_argument("--ref-sample-elems", type=int, default=1_048_576)
+    ap.add_argument("--ref-sample-elems", type=int, default=524_288)
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
