@@ -18,6 +18,12 @@ constexpr int CHUNK = 256;  // elements covered by one warp-wide 256-bit load
 #ifndef QESGD_ENCODE_CHUNKS
 #define QESGD_ENCODE_CHUNKS 4  // chunks per warp in the encode kernel (2 or 4)
 #endif
+#ifndef QESGD_DAA_THREADS
+#define QESGD_DAA_THREADS 128   // threads per CTA of the decode-average-apply kernel
+#endif
+#ifndef QESGD_DAA_MIN_CTAS
+#define QESGD_DAA_MIN_CTAS 5    // resident CTAs per SM its register budget is set for
+#endif
 #ifndef QESGD_ENCODE_MIN_WARPS
 #define QESGD_ENCODE_MIN_WARPS 24  // resident warps per SM the register budget is set for
 #endif
@@ -498,12 +504,32 @@ __device__ __forceinline__ uint32_t and_xor(uint32_t a, uint32_t b, uint32_t c)
 
 // acc += +-level * step for the 8 codes of one octet, two elements per arithmetic
 // instruction (acc[p] holds elements 2p, 2p+1).  One rounding per product-sum: the sign
-// is folded into the multiplier.  Levels are spliced into the mantissa of 2^23 and the
-// 2^23 is subtracted again, which converts them to float exactly.
+// is folded into the multiplier.  `cw` is the 64-bit code word of the lane and `o` the
+// octet inside it (8/BITS octets per word).
 template <int BITS>
-__device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], float step,
+__device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], int o, float step,
                                                  uint64_t (&acc)[4])
 {
+    if (BITS == 2) {
+        // Two-bit codes are (sign, level) with level in {0, 1}.  Moved to bits 31 and 30
+        // they ARE the floats +-2.0 (level 1) and +-0.0 (level 0): bit 31 is the sign and
+        // bit 30 the top exponent bit.  So a shift and a mask decode a code, and multiplying
+        // by step/2 (exact: steps are far above the subnormal range) gives +-step or 0.
+        const uint32_t hs = __float_as_uint(__fmul_rn(step, 0.5f));
+        const uint64_t hs2 = pack2(hs, hs);
+        const uint32_t word = cw[o >> 1];
+        const int base = 16 * (o & 1);           // bit offset of the octet inside the word
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+            const int s0 = 30 - base - 4 * p, s1 = 28 - base - 4 * p;   // left shifts; < 0 = right
+            const uint32_t f0 = (s0 >= 0 ? word << (s0 >= 0 ? s0 : 0) : word >> (s0 < 0 ? -s0 : 0));
+            const uint32_t f1 = (s1 >= 0 ? word << (s1 >= 0 ? s1 : 0) : word >> (s1 < 0 ? -s1 : 0));
+            acc[p] = fma2(pack2(f0 & 0xC0000000u, f1 & 0xC0000000u), hs2, acc[p]);
+        }
+        return;
+    }
+    // Levels are spliced into the mantissa of 2^23 and the 2^23 is subtracted again, which
+    // converts them to float exactly.
     const uint32_t sb = __float_as_uint(step);
     const uint64_t neg_magic = pack2(0xCB000000u, 0xCB000000u);   // (-2^23, -2^23)
     uint32_t m[8], sg[8];
@@ -519,11 +545,11 @@ __device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], float 
             }
         }
     } else {
-        constexpr uint32_t LEVEL_MASK = (1u << (BITS - 1)) - 1u;
+        const uint32_t word = cw[o];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            m[j] = and_or(cw[0] >> (j * BITS), LEVEL_MASK, 0x4B000000u);
-            sg[j] = and_xor(cw[0] << (31 - (j * BITS + BITS - 1)), 0x80000000u, sb);
+            m[j] = and_or(word >> (j * 4), 7u, 0x4B000000u);
+            sg[j] = and_xor(word << (28 - j * 4), 0x80000000u, sb);
         }
     }
 #pragma unroll
@@ -532,90 +558,114 @@ __device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], float 
                       pack2(sg[2 * p], sg[2 * p + 1]), acc[p]);
 }
 
-// One octet per lane, one chunk of 256 elements per warp.  The K grid spacings
-// fl32(scale/s) a chunk needs are computed once per warp (one division per lane)
-// and handed out by shuffle; code words are fetched eight workers at a time so that
-// eight independent loads are in flight per lane before the first is used.
+// Every lane owns 8/BITS consecutive octets -- exactly one 64-bit code word per worker --
+// and a warp 256 * 8/BITS consecutive elements.  The grid spacings fl32(scale/s) a warp
+// needs are computed once per warp (one division per lane) and handed out by shuffle;
+// code words are fetched several workers at a time so that independent loads are in
+// flight before the first is used.
 template <int BITS, bool VEC>
-__global__ void __launch_bounds__(256) qesgd_decode_average_apply_kernel(const DecodeArgs a)
+__global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
+    qesgd_decode_average_apply_kernel(const DecodeArgs a)
 {
-    constexpr int BATCH = 8;
+    constexpr int OPL = 8 / BITS;                 // octets per lane: 4, 2, 1
+    constexpr int LANE_ELEMS = 8 * OPL;
+    constexpr uint32_t WCHUNK = 32 * LANE_ELEMS;  // elements per warp: 1024, 512, 256
+    constexpr uint32_t LOG2_WCHUNK = BITS == 2 ? 10 : (BITS == 4 ? 9 : 8);
+    constexpr int BATCH = 4;
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp_eb =
-        (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * (uint64_t)CHUNK;
+        (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * (uint64_t)WCHUNK;
     if (warp_eb >= a.d) return;  // whole warp out of range
-    const uint64_t eb = warp_eb + lane * 8u;
+    const uint64_t eb = warp_eb + lane * (uint32_t)LANE_ELEMS;
     const uint32_t lb = a.log2_bucket;
-    const uint32_t nbw = lb >= 8 ? 1u : (uint32_t)CHUNK >> lb;  // buckets per chunk: 1, 2, 4
-    const uint32_t sub = lb >= 8 ? 0u : (lane * 8u) >> lb;      // this lane's bucket in the chunk
+    const uint32_t nbw = lb >= LOG2_WCHUNK ? 1u : WCHUNK >> lb;          // buckets per warp: 1..16
+    const uint32_t sub = lb >= LOG2_WCHUNK ? 0u : (lane * (uint32_t)LANE_ELEMS) >> lb;
     const uint64_t bucket0 = warp_eb >> lb;
-    const uint32_t per_pass = 32u / nbw;                        // workers per pass
+    const uint32_t per_pass = 32u / nbw;                                 // workers per pass
     const float sf = (float)a.s;
-    const bool vec_ok = VEC && eb + 8 <= a.d;
 
-    float w[8];
-    if (vec_ok) {
-        ld256_rw(a.param + eb, w);
-    } else {
+    float w[OPL][8];
 #pragma unroll
-        for (int j = 0; j < 8; ++j) w[j] = (eb + j < a.d) ? a.param[eb + j] : 0.0f;
+    for (int o = 0; o < OPL; ++o) {
+        const uint64_t e0 = eb + 8u * o;
+        if (VEC && e0 + 8 <= a.d) {
+            ld256_rw(a.param + e0, w[o]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[o][j] = (e0 + j < a.d) ? a.param[e0 + j] : 0.0f;
+        }
     }
-    uint64_t acc[4] = {0ull, 0ull, 0ull, 0ull};   // four pairs of +0.0f
+    uint64_t acc[OPL][4];
+#pragma unroll
+    for (int o = 0; o < OPL; ++o)
+#pragma unroll
+        for (int p = 0; p < 4; ++p) acc[o][p] = 0ull;   // pairs of +0.0f
 
-    // Lanes past the padded length of the streams read the warp's first octet instead
-    // (their result is never stored), so no load needs a predicate.
+    // Lanes past the padded length of the streams read the warp's first word instead
+    // (their result is never stored), so no load needs a predicate.  The padded length
+    // is a multiple of 64, so a lane's 8, 16 or 32 elements are inside it or outside it.
     const uint64_t safe_eb = eb < (a.nb << lb) ? eb : warp_eb;
     const uint8_t *__restrict__ cp =
         reinterpret_cast<const uint8_t *>(a.codes) + (safe_eb >> 3) * (uint64_t)BITS;
 
-    for (uint32_t k0 = 0; k0 < a.K; k0 += per_pass) {
-        const uint32_t kk = k0 + lane / nbw;
-        const uint64_t bb = bucket0 + (lane % nbw);
-        float st = 0.0f;
-        if (kk < a.K && bb < a.nb)
-            st = __fdiv_rn(__ldg(a.scales + (uint64_t)kk * a.scale_stride + bb), sf);
-        const uint32_t count = min(per_pass, a.K - k0);
-        for (uint32_t i0 = 0; i0 < count; i0 += BATCH) {
-            uint32_t cw[BATCH][2];
+    // Code words of BATCH workers are requested one batch ahead of the batch being decoded.
+    auto fetch = [&](uint32_t kfirst, uint32_t (&dst)[BATCH][2]) {
 #pragma unroll
-            for (int i = 0; i < BATCH; ++i) {
-                cw[i][0] = cw[i][1] = 0u;
-                if (i0 + i < count) {
-                    const uint8_t *q = cp + (uint64_t)(k0 + i0 + i) * a.code_stride;
-                    if (BITS == 8) {
-                        const uint2 v = __ldg(reinterpret_cast<const uint2 *>(q));
-                        cw[i][0] = v.x;
-                        cw[i][1] = v.y;
-                    } else if (BITS == 4) {
-                        cw[i][0] = __ldg(reinterpret_cast<const uint32_t *>(q));
-                    } else {
-                        cw[i][0] = __ldg(reinterpret_cast<const uint16_t *>(q));
-                    }
-                }
+        for (int i = 0; i < BATCH; ++i) {
+            dst[i][0] = dst[i][1] = 0u;
+            if (kfirst + i < a.K) {
+                const uint2 v = __ldg(reinterpret_cast<const uint2 *>(
+                    cp + (uint64_t)(kfirst + i) * a.code_stride));
+                dst[i][0] = v.x;
+                dst[i][1] = v.y;
             }
+        }
+    };
+    uint32_t cw[BATCH][2], nx[BATCH][2];
+    fetch(0u, cw);
+    float st = 0.0f;
+    for (uint32_t kb = 0; kb < a.K; kb += BATCH) {
+        fetch(kb + BATCH, nx);
 #pragma unroll
-            for (int i = 0; i < BATCH; ++i) {
-                if (i0 + i < count) {   // uniform across the warp
-                    const float step = __shfl_sync(FULL, st, (i0 + i) * nbw + sub);
-                    accumulate_octet<BITS>(cw[i], step, acc);
+        for (int i = 0; i < BATCH; ++i) {
+            const uint32_t k = kb + i;
+            if (k < a.K) {   // uniform across the warp
+                if (k % per_pass == 0u) {   // a new pass: every lane computes one spacing
+                    const uint32_t kk = k + lane / nbw;
+                    const uint64_t bb = bucket0 + (lane % nbw);
+                    st = 0.0f;
+                    if (kk < a.K && bb < a.nb)
+                        st = __fdiv_rn(__ldg(a.scales + (uint64_t)kk * a.scale_stride + bb), sf);
                 }
+                const float step = __shfl_sync(FULL, st, (k % per_pass) * nbw + sub);
+#pragma unroll
+                for (int o = 0; o < OPL; ++o) accumulate_octet<BITS>(cw[i], o, step, acc[o]);
             }
+        }
+#pragma unroll
+        for (int i = 0; i < BATCH; ++i) {
+            cw[i][0] = nx[i][0];
+            cw[i][1] = nx[i][1];
         }
     }
     const float inv_k = __fdiv_rn(1.0f, (float)a.K);
 #pragma unroll
-    for (int p = 0; p < 4; ++p) {
-        float lo, hi;
-        unpack2(acc[p], lo, hi);
-        w[2 * p] = __fmaf_rn(lo, inv_k, w[2 * p]);
-        w[2 * p + 1] = __fmaf_rn(hi, inv_k, w[2 * p + 1]);
-    }
-    if (vec_ok) {
-        st256(a.param + eb, w);
-    } else {
+    for (int o = 0; o < OPL; ++o) {
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if (eb + j < a.d) a.param[eb + j] = w[j];
+        for (int p = 0; p < 4; ++p) {
+            float lo, hi;
+            unpack2(acc[o][p], lo, hi);
+            w[o][2 * p] = __fmaf_rn(lo, inv_k, w[o][2 * p]);
+            w[o][2 * p + 1] = __fmaf_rn(hi, inv_k, w[o][2 * p + 1]);
+        }
+        const uint64_t e0 = eb + 8u * o;
+        if (VEC && e0 + 8 <= a.d) {
+            st256(a.param + e0, w[o]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (e0 + j < a.d) a.param[e0 + j] = w[o][j];
+        }
     }
 }
 
@@ -698,10 +748,12 @@ int qesgd_launch_decode(const DecodeArgs &a, uint32_t bits, bool vec, cudaStream
 int qesgd_launch_decode_average_apply(const DecodeArgs &a, uint32_t bits, bool vec,
                                       cudaStream_t stream)
 {
-    const uint64_t chunks = (a.d + CHUNK - 1) / CHUNK;  // one warp each
-    const uint64_t blocks = (chunks + 7) / 8;
+    const uint64_t warp_elems = 256ull * (8u / bits);   // one warp each (see the kernel)
+    const uint64_t warps = (a.d + warp_elems - 1) / warp_elems;
+    const uint64_t wpc = QESGD_DAA_THREADS / 32;
+    const uint64_t blocks = (warps + wpc - 1) / wpc;
     if (blocks == 0 || blocks > 0x7FFFFFFFull) return (int)cudaErrorInvalidValue;
-    dim3 grid((unsigned)blocks), block(256);
+    dim3 grid((unsigned)blocks), block(QESGD_DAA_THREADS);
 #define QESGD_DAA(B)                                                                          \
     if (vec) qesgd_decode_average_apply_kernel<B, true><<<grid, block, 0, stream>>>(a);       \
     else qesgd_decode_average_apply_kernel<B, false><<<grid, block, 0, stream>>>(a)
