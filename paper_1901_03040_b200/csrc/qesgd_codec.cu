@@ -19,10 +19,10 @@ constexpr int CHUNK = 256;  // elements covered by one warp-wide 256-bit load
 #define QESGD_ENCODE_CHUNKS 4  // chunks per warp in the encode kernel (2 or 4)
 #endif
 #ifndef QESGD_DAA_THREADS
-#define QESGD_DAA_THREADS 128   // threads per CTA of the decode-average-apply kernel
+#define QESGD_DAA_THREADS 32    // threads per CTA of the decode-average-apply kernel
 #endif
 #ifndef QESGD_DAA_MIN_CTAS
-#define QESGD_DAA_MIN_CTAS 5    // resident CTAs per SM its register budget is set for
+#define QESGD_DAA_MIN_CTAS 16   // resident CTAs per SM its register budget is set for
 #endif
 #ifndef QESGD_ENCODE_MIN_WARPS
 #define QESGD_ENCODE_MIN_WARPS 24  // resident warps per SM the register budget is set for
