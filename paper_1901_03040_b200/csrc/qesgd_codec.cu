@@ -318,24 +318,41 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
     }
 
     // ---- rounding, packing, stores ---------------------------------------------
-    uint8_t *__restrict__ codes = reinterpret_cast<uint8_t *>(a.codes) + (uint64_t)k * a.code_stride;
-    float *__restrict__ scales = a.scales + (uint64_t)k * a.scale_stride;
+    // All addresses of the tile derive from three values computed once; inside the
+    // chunk loop only small compile-time offsets are added.  warp_base is a multiple of
+    // V*256, so the Philox block index (warp_base/8 + lane + 32c) never carries into
+    // its high word when c advances.
+    const uint32_t loff = lane * 8u;
+    uint8_t *const cbase = reinterpret_cast<uint8_t *>(a.codes) + (uint64_t)k * a.code_stride +
+                           ((warp_base + loff) >> 3) * (uint64_t)BITS;
+    float *const sbase = a.scales + (uint64_t)k * a.scale_stride + (warp_base >> lb);
+    const uint64_t blk0 = (warp_base >> 3) + lane;
+    const uint32_t blk_lo = (uint32_t)blk0, blk_hi = (uint32_t)(blk0 >> 32);
     const uint32_t bucket_mask = (1u << lb) - 1u;
+    const bool wide = lb > LOG2_WARP_ELEMS;                     // bucket spans several warps
+    const bool wide_first = ((uint32_t)warp_base & bucket_mask) == 0u;   // this warp starts it
+    const uint32_t wid = a.worker0 + k;
 
 #pragma unroll
     for (int c = 0; c < V; ++c) {
-        const uint64_t eb = warp_base + (uint64_t)c * CHUNK + lane * 8u;
+        const uint32_t off = (uint32_t)c * CHUNK + loff;        // element offset inside the tile
+        const bool inside = FULL || warp_base + off < a.padded;
         float scale = my_scale, inv = my_inv;
         if (MODE != 2) {   // fetch chunk c's bucket scale from the neighbour lane that carried it
             const int src = (int)lane_of_chunk<V>(lane, c);
             scale = __shfl_sync(FULL, my_scale, src);
             inv = __shfl_sync(FULL, my_inv, src);
         }
-        if ((FULL || eb < a.padded) && ((uint32_t)eb & bucket_mask) == 0u) scales[eb >> lb] = scale;
+        if (inside) {      // the first lane of every bucket writes its scale
+            if (!wide) {
+                if ((off & bucket_mask) == 0u) sbase[off >> lb] = scale;
+            } else if (off == 0u && wide_first) {
+                sbase[0] = scale;
+            }
+        }
 
         uint32_t x[4];
-        const uint64_t blk = eb >> 3;
-        philox4x32_10((uint32_t)blk, (uint32_t)(blk >> 32), a.worker0 + k, a.epoch, a.round_key, x);
+        philox4x32_10(blk_lo + 32u * c, blk_hi, wid, a.epoch, a.round_key, x);
 
         uint32_t X[8], Z[8];
 #pragma unroll
@@ -348,13 +365,14 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
         }
         uint32_t out[2];
         pack_octet<BITS>(X, Z, out);
-        if (FULL || eb < a.padded) {
+        if (inside) {
+            uint8_t *const q = cbase + c * (CHUNK * BITS / 8);
             if (BITS == 8) {
-                *reinterpret_cast<uint2 *>(codes + eb) = make_uint2(out[0], out[1]);
+                *reinterpret_cast<uint2 *>(q) = make_uint2(out[0], out[1]);
             } else if (BITS == 4) {
-                *reinterpret_cast<uint32_t *>(codes + (eb >> 1)) = out[0];
+                *reinterpret_cast<uint32_t *>(q) = out[0];
             } else {
-                *reinterpret_cast<uint16_t *>(codes + (eb >> 2)) = (uint16_t)out[0];
+                *reinterpret_cast<uint16_t *>(q) = (uint16_t)out[0];
             }
         }
     }
