@@ -93,6 +93,55 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
     x[0] = c0; x[1] = c1; x[2] = c2; x[3] = c3;
 }
 
+// ------------------------------------------------- packed fp32 pairs --------
+// sm_100 adds add / sub / mul / fma on two floats held in a 64-bit register pair.
+__device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi)
+{
+    uint64_t p;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p) : "r"(lo), "r"(hi));
+    return p;
+}
+__device__ __forceinline__ uint64_t pack2f(float lo, float hi)
+{
+    uint64_t p;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(p) : "f"(lo), "f"(hi));
+    return p;
+}
+__device__ __forceinline__ void unpack2(uint64_t p, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b)
+{
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t fma2_ru(uint64_t a, uint64_t b, uint64_t c)   // toward +inf
+{
+    uint64_t d;
+    asm("fma.rp.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
 // ------------------------------------------------------- rounding (Eq. 4) ----
 // level = floor(r) + [h + 1/2 < frac(r) * 2^16] for r = min(|z|*inv, s), 0 <= r <= 127.
 //
@@ -104,11 +153,21 @@ __device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t
 // r = 0 (where the sum would be 2^23 - 1/2 exactly, below the integer binade)
 // gives U = 0 like every r with r * 2^16 <= 1/2; the same clamp turns the NaN of
 // an invalid bucket (inv = 0) into level 0.
-__device__ __forceinline__ uint32_t level_times_65536(float a, float inv, float sf, uint32_t h)
+// Two neighbouring elements at a time: the multiply and the fused multiply-add run on
+// packed pairs, the clamp stays scalar (it takes |.| for free).  x0, x1 receive the level
+// in bits 16..22 (what is below is of no interest).
+__device__ __forceinline__ void level_pair(float z0, float z1, uint64_t inv2, float sf,
+                                           uint32_t h0, uint32_t h1, uint32_t &x0, uint32_t &x1)
 {
-    const float r = fminf(fmaxf(__fmul_rn(a, inv), 0x1p-30f), sf);
-    const uint32_t ub = __float_as_uint(__fmaf_ru(r, 65536.0f, 8388607.5f));
-    return ub - h + (65535u - 0x4B000000u);   // level in bits 16..22, below: don't care
+    float t0, t1;
+    unpack2(mul2(pack2f(z0, z1), inv2), t0, t1);           // sign rides along, removed by |.|
+    const float r0 = fminf(fmaxf(fabsf(t0), 0x1p-30f), sf);
+    const float r1 = fminf(fmaxf(fabsf(t1), 0x1p-30f), sf);
+    float u0, u1;
+    unpack2(fma2_ru(pack2f(r0, r1), pack2f(65536.0f, 65536.0f), pack2f(8388607.5f, 8388607.5f)),
+            u0, u1);
+    x0 = __float_as_uint(u0) - h0 + (65535u - 0x4B000000u);
+    x1 = __float_as_uint(u1) - h1 + (65535u - 0x4B000000u);
 }
 
 // Packing.  X[j] holds the level of element j in byte 2 (bits 16..22) and Z[j] the
@@ -355,13 +414,15 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
         philox4x32_10(blk_lo + 32u * c, blk_hi, wid, a.epoch, a.round_key, x);
 
         uint32_t X[8], Z[8];
+        const uint64_t inv2 = pack2f(inv, inv);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            const uint32_t h = (j & 1) ? (x[j >> 1] >> 16) : (x[j >> 1] & 0xFFFFu);
+        for (int j = 0; j < 8; j += 2) {
             Z[j] = __float_as_uint(z[c][j]);
+            Z[j + 1] = __float_as_uint(z[c][j + 1]);
             if (MODE == 2)   // NaN has no place on the grid: flagged (and encoded as 0 by the clamp)
-                flag |= (Z[j] & 0x7FFFFFFFu) > 0x7F800000u;
-            X[j] = level_times_65536(fabsf(z[c][j]), inv, sf, h);
+                flag |= (Z[j] & 0x7FFFFFFFu) > 0x7F800000u || (Z[j + 1] & 0x7FFFFFFFu) > 0x7F800000u;
+            level_pair(z[c][j], z[c][j + 1], inv2, sf, x[j >> 1] & 0xFFFFu, x[j >> 1] >> 16,
+                       X[j], X[j + 1]);
         }
         uint32_t out[2];
         pack_octet<BITS>(X, Z, out);
@@ -409,7 +470,9 @@ __global__ void __launch_bounds__(WARPS * 32, QESGD_ENCODE_MIN_WARPS / WARPS)
 #pragma unroll
             for (int c = 0; c < V; ++c)
 #pragma unroll
-                for (int j = 0; j < 8; ++j) z[c][j] = __fsub_rn(z[c][j], w[c][j]);
+                for (int j = 0; j < 8; j += 2)
+                    unpack2(sub2(pack2f(z[c][j], z[c][j + 1]), pack2f(w[c][j], w[c][j + 1])),
+                            z[c][j], z[c][j + 1]);
         }
         encode_warp_tile<BITS, MODE, V, true>(a, z, warp_base, k, lane, warp, sh, 0u);
         return;
@@ -483,29 +546,6 @@ __global__ void __launch_bounds__(256) qesgd_decode_kernel(const DecodeArgs a)
 }
 
 // -------------------------------------------- decode + average + apply ------
-// Packed fp32 pairs (sm_100: add/fma on two floats per instruction).
-__device__ __forceinline__ uint64_t pack2(uint32_t lo, uint32_t hi)
-{
-    uint64_t p;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(p) : "r"(lo), "r"(hi));
-    return p;
-}
-__device__ __forceinline__ void unpack2(uint64_t p, float &lo, float &hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p));
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b)
-{
-    uint64_t d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c)
-{
-    uint64_t d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
 // (a & b) | c and (a & b) ^ c as one three-input logic operation each
 __device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c)
 {
