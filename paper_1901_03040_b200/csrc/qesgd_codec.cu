@@ -666,6 +666,13 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
     const uint8_t *__restrict__ cp =
         reinterpret_cast<const uint8_t *>(a.codes) + (safe_eb >> 3) * (uint64_t)BITS;
 
+    // Four-bit codes with buckets of at least 256 elements: a half-warp (16 lanes x 16
+    // elements) lies inside one bucket, so the 16 possible code values +-level * step of a
+    // worker fit one per lane and decoding becomes a 16-wide shuffle.  signed_level is the
+    // level of code (lane & 15) with its sign: 0..7, -0..-7.
+    const bool lut = BITS == 4 && lb >= 8;
+    const float signed_level = (lane & 8u) ? -(float)(lane & 7u) : (float)(lane & 7u);
+
     // Code words of BATCH workers are requested one batch ahead of the batch being decoded.
     auto fetch = [&](uint32_t kfirst, uint32_t (&dst)[BATCH][2]) {
 #pragma unroll
@@ -696,8 +703,24 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
                         st = __fdiv_rn(__ldg(a.scales + (uint64_t)kk * a.scale_stride + bb), sf);
                 }
                 const float step = __shfl_sync(FULL, st, (k % per_pass) * nbw + sub);
+                if (BITS == 4 && lut) {
+                    // every lane holds the value of code (lane & 15) for this worker; a code
+                    // is decoded by fetching its value from that lane of the same half-warp
+                    const float tab = __fmul_rn(signed_level, step);
 #pragma unroll
-                for (int o = 0; o < OPL; ++o) accumulate_octet<BITS>(cw[i], o, step, acc[o]);
+                    for (int o = 0; o < OPL; ++o) {
+                        const uint32_t word = cw[i][o];
+#pragma unroll
+                        for (int p = 0; p < 4; ++p) {
+                            const float v0 = __shfl_sync(FULL, tab, (int)(word >> (8 * p)), 16);
+                            const float v1 = __shfl_sync(FULL, tab, (int)(word >> (8 * p + 4)), 16);
+                            acc[o][p] = add2(acc[o][p], pack2f(v0, v1));
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int o = 0; o < OPL; ++o) accumulate_octet<BITS>(cw[i], o, step, acc[o]);
+                }
             }
         }
 #pragma unroll
