@@ -21,6 +21,9 @@ constexpr int CHUNK = 256;  // elements covered by one warp-wide 256-bit load
 #ifndef QESGD_DAA_THREADS
 #define QESGD_DAA_THREADS 32    // threads per CTA of the decode-average-apply kernel
 #endif
+#ifndef QESGD_DAA_BATCH
+#define QESGD_DAA_BATCH 4       // workers whose code words are fetched together
+#endif
 #ifndef QESGD_DAA_MIN_CTAS
 #define QESGD_DAA_MIN_CTAS 16   // resident CTAs per SM its register budget is set for
 #endif
@@ -629,7 +632,7 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
     constexpr int LANE_ELEMS = 8 * OPL;
     constexpr uint32_t WCHUNK = 32 * LANE_ELEMS;  // elements per warp: 1024, 512, 256
     constexpr uint32_t LOG2_WCHUNK = BITS == 2 ? 10 : (BITS == 4 ? 9 : 8);
-    constexpr int BATCH = 4;
+    constexpr int BATCH = QESGD_DAA_BATCH;
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp_eb =
         (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * (uint64_t)WCHUNK;
