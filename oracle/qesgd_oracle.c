@@ -96,13 +96,20 @@ static double tree_sum(const double *x, size_t n)
     return tree_sum(x, n / 2) + tree_sum(x + n / 2, n / 2);
 }
 
+/* The fp64 sum of squares of one zero-padded bucket, before the square root (exposed so
+ * that tests can check the summation tree in fp64, where its shape is visible). */
+double qesgd_ref_bucket_sumsq(const float *z, uint32_t B, double *scratch)
+{
+    for (uint32_t j = 0; j < B; ++j)
+        scratch[j] = (double)z[j] * (double)z[j]; /* exact: 24-bit x 24-bit */
+    return tree_sum(scratch, B);
+}
+
 /* z holds one zero-padded bucket of B = 2^m fp32 values. */
 float qesgd_ref_bucket_scale(const float *z, uint32_t B, uint32_t scale_mode, double *scratch)
 {
     if (scale_mode == QREF_SCALE_NORM) {
-        for (uint32_t j = 0; j < B; ++j)
-            scratch[j] = (double)z[j] * (double)z[j]; /* exact: 24-bit x 24-bit */
-        double S = tree_sum(scratch, B);
+        double S = qesgd_ref_bucket_sumsq(z, B, scratch);
         return (float)sqrt(S); /* fl32(fl64(sqrt(S))) */
     }
     float m = 0.0f;

@@ -25,6 +25,8 @@ _lib.qesgd_ref_draw16.argtypes = [_u64, _u32, _u32, _u64]
 _lib.qesgd_ref_draw16.restype = _u32
 _lib.qesgd_ref_bucket_scale.argtypes = [_pf, _u32, _u32, _pd]
 _lib.qesgd_ref_bucket_scale.restype = _f32
+_lib.qesgd_ref_bucket_sumsq.argtypes = [_pf, _u32, _pd]
+_lib.qesgd_ref_bucket_sumsq.restype = C.c_double
 _lib.qesgd_ref_level.argtypes = [_f32, _f32, _u32, _u32]
 _lib.qesgd_ref_level.restype = _u32
 _lib.qesgd_ref_num_buckets.argtypes = [_u64, _u32]
@@ -79,6 +81,12 @@ def bucket_scale(z, scale_mode):
     scratch = np.zeros(z.size, dtype=np.float64)
     return np.float32(_lib.qesgd_ref_bucket_scale(_f(z), z.size, scale_mode,
                                                   scratch.ctypes.data_as(_pd)))
+
+
+def bucket_sumsq(z):
+    z = np.ascontiguousarray(z, dtype=np.float32)
+    scratch = np.zeros(z.size, dtype=np.float64)
+    return float(_lib.qesgd_ref_bucket_sumsq(_f(z), z.size, scratch.ctypes.data_as(_pd)))
 
 
 def level(a, inv, s, h):

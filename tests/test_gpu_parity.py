@@ -135,6 +135,27 @@ def test_fixed_delta_mode_matches_and_clips():
         assert got[2] == qesgd.STATUS_NONFINITE
 
 
+def test_negative_zero_and_exact_ties_match_the_oracle():
+    """Values whose fractional part times 2^16 is a half-integer sit exactly on the
+    boundary between two draws (h + 1/2 = p * 2^16): strict '<' must decide them the same
+    way on both sides; negative values that round to level 0 must give the plain 0 code."""
+    s, bits, bucket = 7, 4, 64
+    delta = 2.0 ** -4
+    z = np.zeros(bucket * 2, dtype=np.float32)
+    z[0] = s * delta                                   # scale = s * delta, inv = 16 exactly
+    ties = [(2 * m + 1) / 131072.0 for m in (0, 1, 5, 1000, 32767, 65535)]
+    for n, t in enumerate(ties):
+        z[1 + n] = (n % 7 + t) * delta * (-1 if n % 2 else 1)
+    z[10:40] = -1e-9
+    z[40] = -0.0
+    z[64] = -s * delta
+    z[65:] = z[1:64]
+    for epoch in range(8):
+        args = (bucket, s, bits, ref.SCALE_MAX, 31337, 2, epoch)
+        got, want = G.gpu_encode(z, None, *args), ref.encode(z, None, *args)
+        _assert_streams_equal(got, want)
+
+
 def test_on_grid_input_round_trips_exactly_on_the_gpu():
     s, bits, bucket = 127, 8, 256
     rng = np.random.default_rng(4)

@@ -63,7 +63,8 @@ def _levels_over_all_draws(a, inv, s):
 
 
 @pytest.mark.parametrize("v_over_delta", ["0", "1/3", "5/2", "6.999", "7", "2.0000305", "0.5",
-                                          "3.99999", "1e-7", "6.25"])
+                                          "3.99999", "1e-7", "6.25", "262147/131072",
+                                          "65535/131072", "1/131072"])
 def test_rounding_probability_matches_eq4(v_over_delta):
     """P(ceil) = (v - delta*floor(v/delta))/delta, P(floor) = 1 - that (Eq. 4),
     realised with 16-bit draws: the count of 'up' draws is exactly the number of
@@ -143,6 +144,7 @@ def test_norm_scale_uses_balanced_tree():
             x = x[0::2] + x[1::2]
         tree = np.float32(np.sqrt(x[0]))
         assert q.bucket_scale(z, q.SCALE_NORM) == tree
+        assert q.bucket_sumsq(z) == float(x[0])      # the fp64 sum itself, bit for bit
         differs += float(x[0]) != seq
     assert differs > 0   # the test can tell a tree from a running sum
 
@@ -199,6 +201,19 @@ def test_grid_points_are_fixed_points_for_every_seed(bits):
     assert (_signed_levels(codes, k.size, bits) == k).all()
     assert sorted(set(_unpack(codes, 512, bits).tolist())) == \
         sorted(set(range(0, s + 1)) | set(range((1 << (bits - 1)) + 1, (1 << (bits - 1)) + s + 1)))
+
+
+def test_no_negative_zero_code():
+    """A negative value that rounds to level 0 is encoded as plain 0: the grid has one zero."""
+    for bits, s in ((2, 1), (4, 7), (8, 127)):
+        z = np.zeros(64, dtype=np.float32)
+        z[0] = 1.0
+        z[1:40] = -1e-9          # level 0 for every draw that matters
+        z[40] = -0.0
+        for seed in range(4):
+            codes, scales, _ = q.encode(z, None, 64, s, bits, q.SCALE_MAX, seed, 0, 0)
+            c = _unpack(codes, 64, bits)
+            assert c[0] == s and (c[1:] == 0).all()
 
 
 def test_norm_mode_single_nonzero_is_exact():
