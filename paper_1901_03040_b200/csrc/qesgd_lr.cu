@@ -6,8 +6,8 @@
 //           keeps its slice of u in registers and writes sum_{cols} x_jc u_c for every
 //           row j to work[(k*P + p)*m + j]   (no atomics, fixed summation order)
 //   pass 2  every CTA sums the P partials of each row, forms the step coefficients
-//           (lr/m) * y_j / (1 + exp(y_j m_j)) in shared memory and updates 512 columns
-//           of u with sum_j coef_j x_jc.  X_B is normally still in L2 for this pass.
+//           (lr/m) * y_j / (1 + exp(y_j m_j)) in shared memory and updates 256 columns
+//           of u with sum_j coef_j x_jc, the rows split over four thread groups.  X_B is normally still in L2 for this pass.
 // No tensor cores: with m = 64 rows the work is 64 dot products, bound by memory.
 #include <mutex>
 
@@ -17,7 +17,9 @@ namespace {
 
 constexpr int SEG = 1024;        // columns per segment in pass 1 (32 lanes x 8 float4)
 constexpr int MAX_PARTS = 64;    // partial-margin slots per worker
-constexpr int UPD_THREADS = 128; // pass 2: 4 columns per thread
+constexpr int UPD_COLS = 256;      // pass 2: columns per CTA (64 groups of 4)
+constexpr int UPD_ROWGROUPS = 4;   // pass 2: row groups per CTA
+constexpr int UPD_THREADS = (UPD_COLS / 4) * UPD_ROWGROUPS;
 
 struct LrArgs {
     const float *X;
@@ -60,32 +62,52 @@ __global__ void __launch_bounds__(256) qesgd_lr_margin_kernel(const LrArgs a)
                 uu[i].w = c + 3 < a.d ? u[c + 3] : 0.0f;
             }
         }
-        for (uint32_t j = warp; j < a.m; j += 8) {  // each row belongs to one warp
-            const float *__restrict__ row = X + (uint64_t)j * a.d;
-            float4 xx[8];
+        // each row belongs to one warp; two rows at a time so that 16 loads are in flight
+        // per lane and the two shuffle reductions interleave
+        for (uint32_t j = warp; j < a.m; j += 16) {
+            const uint32_t j2 = j + 8;
+            const bool two = j2 < a.m;
+            const float *__restrict__ row0 = X + (uint64_t)j * a.d;
+            const float *__restrict__ row1 = X + (uint64_t)(two ? j2 : j) * a.d;
+            float4 xa[8], xb[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
                 const uint64_t c = c0 + (uint64_t)i * 128 + lane * 4u;
                 if (VEC && c + 4 <= a.d) {
-                    xx[i] = __ldg(reinterpret_cast<const float4 *>(row + c));
+                    xa[i] = __ldg(reinterpret_cast<const float4 *>(row0 + c));
+                    xb[i] = __ldg(reinterpret_cast<const float4 *>(row1 + c));
                 } else {
-                    xx[i].x = c + 0 < a.d ? __ldg(row + c + 0) : 0.0f;
-                    xx[i].y = c + 1 < a.d ? __ldg(row + c + 1) : 0.0f;
-                    xx[i].z = c + 2 < a.d ? __ldg(row + c + 2) : 0.0f;
-                    xx[i].w = c + 3 < a.d ? __ldg(row + c + 3) : 0.0f;
+                    xa[i].x = c + 0 < a.d ? __ldg(row0 + c + 0) : 0.0f;
+                    xa[i].y = c + 1 < a.d ? __ldg(row0 + c + 1) : 0.0f;
+                    xa[i].z = c + 2 < a.d ? __ldg(row0 + c + 2) : 0.0f;
+                    xa[i].w = c + 3 < a.d ? __ldg(row0 + c + 3) : 0.0f;
+                    xb[i].x = c + 0 < a.d ? __ldg(row1 + c + 0) : 0.0f;
+                    xb[i].y = c + 1 < a.d ? __ldg(row1 + c + 1) : 0.0f;
+                    xb[i].z = c + 2 < a.d ? __ldg(row1 + c + 2) : 0.0f;
+                    xb[i].w = c + 3 < a.d ? __ldg(row1 + c + 3) : 0.0f;
                 }
             }
-            float acc = 0.0f;
+            float acc0 = 0.0f, acc1 = 0.0f;
 #pragma unroll
             for (int i = 0; i < 8; ++i) {
-                acc = fmaf(xx[i].x, uu[i].x, acc);
-                acc = fmaf(xx[i].y, uu[i].y, acc);
-                acc = fmaf(xx[i].z, uu[i].z, acc);
-                acc = fmaf(xx[i].w, uu[i].w, acc);
+                acc0 = fmaf(xa[i].x, uu[i].x, acc0);
+                acc0 = fmaf(xa[i].y, uu[i].y, acc0);
+                acc0 = fmaf(xa[i].z, uu[i].z, acc0);
+                acc0 = fmaf(xa[i].w, uu[i].w, acc0);
+                acc1 = fmaf(xb[i].x, uu[i].x, acc1);
+                acc1 = fmaf(xb[i].y, uu[i].y, acc1);
+                acc1 = fmaf(xb[i].z, uu[i].z, acc1);
+                acc1 = fmaf(xb[i].w, uu[i].w, acc1);
             }
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
-            if (lane == 0) s_part[j] += acc;
+            for (int off = 16; off > 0; off >>= 1) {
+                acc0 += __shfl_xor_sync(0xFFFFFFFFu, acc0, off);
+                acc1 += __shfl_xor_sync(0xFFFFFFFFu, acc1, off);
+            }
+            if (lane == 0) {
+                s_part[j] += acc0;
+                if (two) s_part[j2] += acc1;
+            }
         }
     }
     __syncthreads();
@@ -93,10 +115,14 @@ __global__ void __launch_bounds__(256) qesgd_lr_margin_kernel(const LrArgs a)
     for (uint32_t j = threadIdx.x; j < a.m; j += blockDim.x) out[j] = s_part[j];
 }
 
+// Pass 2.  A CTA updates UPD_COLS consecutive columns: 64 column groups of 4 columns
+// times UPD_ROWGROUPS row groups; row group g sums rows g, g + G, g + 2G, ... (coalesced
+// 1 KB per row), the G partial sums meet in shared memory in fixed order.
 template <bool VEC>
 __global__ void __launch_bounds__(UPD_THREADS) qesgd_lr_update_kernel(const LrArgs a)
 {
     __shared__ float s_coef[QESGD_MAX_LR_BATCH];
+    __shared__ float4 s_sum[UPD_ROWGROUPS][UPD_COLS / 4];
     const uint32_t k = blockIdx.y;
     const float *__restrict__ X = a.X + (uint64_t)k * a.x_stride;
     const float *__restrict__ y = a.y + (uint64_t)k * a.y_stride;
@@ -111,13 +137,14 @@ __global__ void __launch_bounds__(UPD_THREADS) qesgd_lr_update_kernel(const LrAr
     }
     __syncthreads();
 
-    const uint64_t c = ((uint64_t)blockIdx.x * UPD_THREADS + threadIdx.x) * 4u;
-    if (c >= a.d) return;
+    const uint32_t cg = threadIdx.x % (UPD_COLS / 4);     // column group inside the CTA
+    const uint32_t rg = threadIdx.x / (UPD_COLS / 4);     // row group
+    const uint64_t c = (uint64_t)blockIdx.x * UPD_COLS + cg * 4u;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     if (VEC && c + 4 <= a.d) {
         const float *__restrict__ col = X + c;
 #pragma unroll 8
-        for (uint32_t j = 0; j < a.m; ++j) {
+        for (uint32_t j = rg; j < a.m; j += UPD_ROWGROUPS) {
             const float4 x = __ldg(reinterpret_cast<const float4 *>(col + (uint64_t)j * a.d));
             const float cj = s_coef[j];
             acc.x = fmaf(cj, x.x, acc.x);
@@ -125,16 +152,34 @@ __global__ void __launch_bounds__(UPD_THREADS) qesgd_lr_update_kernel(const LrAr
             acc.z = fmaf(cj, x.z, acc.z);
             acc.w = fmaf(cj, x.w, acc.w);
         }
-        float4 uu = *reinterpret_cast<float4 *>(u + c);
-        uu.x += acc.x; uu.y += acc.y; uu.z += acc.z; uu.w += acc.w;
-        *reinterpret_cast<float4 *>(u + c) = uu;
-    } else {
-        for (int e = 0; e < 4; ++e) {
-            if (c + e >= a.d) break;
-            float s = 0.0f;
-            for (uint32_t j = 0; j < a.m; ++j)
-                s = fmaf(s_coef[j], __ldg(X + (uint64_t)j * a.d + c + e), s);
-            u[c + e] += s;
+    } else if (c < a.d) {
+        for (uint32_t j = rg; j < a.m; j += UPD_ROWGROUPS) {
+            const float cj = s_coef[j];
+            const float *__restrict__ row = X + (uint64_t)j * a.d + c;
+            acc.x = fmaf(cj, __ldg(row), acc.x);
+            if (c + 1 < a.d) acc.y = fmaf(cj, __ldg(row + 1), acc.y);
+            if (c + 2 < a.d) acc.z = fmaf(cj, __ldg(row + 2), acc.z);
+            if (c + 3 < a.d) acc.w = fmaf(cj, __ldg(row + 3), acc.w);
+        }
+    }
+    s_sum[rg][cg] = acc;
+    __syncthreads();
+    if (rg == 0 && c < a.d) {
+        float4 t = s_sum[0][cg];
+#pragma unroll
+        for (int g = 1; g < UPD_ROWGROUPS; ++g) {
+            const float4 v = s_sum[g][cg];
+            t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
+        }
+        if (VEC && c + 4 <= a.d) {
+            float4 uu = *reinterpret_cast<float4 *>(u + c);
+            uu.x += t.x; uu.y += t.y; uu.z += t.z; uu.w += t.w;
+            *reinterpret_cast<float4 *>(u + c) = uu;
+        } else {
+            u[c] += t.x;
+            if (c + 1 < a.d) u[c + 1] += t.y;
+            if (c + 2 < a.d) u[c + 2] += t.z;
+            if (c + 3 < a.d) u[c + 3] += t.w;
         }
     }
 }
@@ -169,7 +214,7 @@ int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float 
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return (int)e;
     *launched = 1;
-    const uint64_t ublocks = (d + UPD_THREADS * 4 - 1) / (UPD_THREADS * 4);
+    const uint64_t ublocks = (d + UPD_COLS - 1) / UPD_COLS;
     if (ublocks > 0x7FFFFFFFull) return (int)cudaErrorInvalidValue;
     dim3 g2((unsigned)ublocks, K), b2(UPD_THREADS);
     if (vec) qesgd_lr_update_kernel<true><<<g2, b2, 0, stream>>>(a);
