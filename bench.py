@@ -371,7 +371,9 @@ def run_c2(args, device, world, rank):
     input in L2."""
     import torch
     from paper_1901_03040_b200 import qesgd, synthetic
-    d, B, R = 1 << 24, 512, 4
+    d, B = (args.d or (1 << 24)), 512
+    R = max(4, (256 << 20) // (4 * d) + 1)      # input sets: together larger than L2
+    mode = {"norm": qesgd.SCALE_NORM, "max": qesgd.SCALE_MAX, "fixed": qesgd.SCALE_FIXED}[args.scale_mode]
     stream = torch.cuda.Stream(device)
     ctx = qesgd.Context(device.index, stream)
     zs = [synthetic.device_normal_f32((d,), 1e-3, 10 + r, device) for r in range(R)]
@@ -389,22 +391,25 @@ def run_c2(args, device, world, rank):
             def call(i):
                 codes, scales = bufs[bits][i % R]
                 if kind == "encode":
-                    ctx.qesgd_encode(zs[i % R], None, d, B, s, bits, qesgd.SCALE_NORM, 1, 0, i,
-                                     codes, scales)
+                    ctx.qesgd_encode(zs[i % R], None, d, B, s, bits, mode, 1, 0, i, codes, scales,
+                                     fixed_delta=3e-3 / s)
                 else:
                     ctx.qesgd_decode(codes, scales, d, B, s, bits, outs[i % R])
             for i in range(max(args.warmup, R)):
                 call(i)
             torch.cuda.synchronize()
-            evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
-            evs[0].record(stream)
+            # one event pair around all launches of this kind: per-launch time = total / steps
+            # (back-to-back launches on one stream, no event between them)
+            e0 = torch.cuda.Event(enable_timing=True)
+            e1 = torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
             for i in range(args.steps):
                 call(i)
-                evs[i + 1].record(stream)
+            e1.record(stream)
             torch.cuda.synchronize()
-            ms = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
-            avg = statistics.mean(ms)
-            t_total += sum(ms)
+            avg = e0.elapsed_time(e1) / args.steps
+            ms = [avg]
+            t_total += avg * args.steps
             nbytes = d * (4.0 + bits / 8.0 + 4.0 / B)
             results[f"{kind}_{bits}bit"] = {
                 "avg_ms": avg, "min_ms": min(ms), "hbm_gbs": nbytes / (avg * 1e-3) / 1e9,
@@ -417,9 +422,10 @@ def run_c2(args, device, world, rank):
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": t_total / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": "C2 quantizer microbench: d=2^24 delta ~N(0,1e-3^2), bucket 512, "
-                                   "s in {1,7,127}: encode then decode; 4 rotating input sets (256 MiB) "
-                                   "defeat L2"},
+            "config": {"workload": "C2 quantizer microbench: delta ~N(0,1e-3^2), bucket 512, "
+                                   "s in {1,7,127}: encode then decode; rotating input sets larger "
+                                   "than L2 together", "d": d, "input_sets": R,
+                       "scale_mode": args.scale_mode},
             "gpu_launches": int(ctx.qesgd_launch_count() - launches0),
             "roofline": {"bound": "hbm", "kernel": "qesgd_encode_kernel (4-bit, no anchor)",
                          "achieved": enc["hbm_gbs"], "peak": peak, "unit": "GB/s",
@@ -548,6 +554,9 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=["c4", "c3", "c5", "c2", "c1"], default="c4")
     ap.add_argument("--bucket", type=int, default=0, help="override the bucket size (c5 sweep)")
+    ap.add_argument("--d", type=int, default=0, help="vector length for --workload c2")
+    ap.add_argument("--scale-mode", choices=["norm", "max", "fixed"], default="norm",
+                    help="bucket scale of --workload c2")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-sample-elems", type=int, default=12_778_496)
