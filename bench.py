@@ -80,7 +80,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(gpu_index), "--query-gpu=" + self.QUERY,
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
@@ -511,7 +511,10 @@ def run_reference(args):
     if args.bucket:
         w["bucket"] = args.bucket
     d, K, bits, s, B = w["d"], w["K"], w["bits"], w["s"], w["bucket"]
-    n = min(d, args.ref_sample_elems // B * B)
+    # the sample shrinks with the number of steps so that the whole run takes about a minute
+    # (the oracle encodes roughly 3e7 elements per second on one core)
+    budget = int(1.4e9 / (K * (args.steps + args.warmup)))
+    n = max(8 * B, min(d, args.ref_sample_elems, budget) // B * B)
     anchor = synthetic.anchor_vector(n, seed=1)
     locs = synthetic.worker_locals(anchor, K, w["sigma"], seed=2, outlier_prob=w["outlier"])
     param = anchor.copy()
@@ -549,7 +552,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--workload", choices=["c4", "c3", "c5", "c2", "c1"], default="c4")
@@ -559,8 +562,8 @@ def main():
                     help="bucket scale of --workload c2")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
-    ap.add_argument("--cpu-sample-elems", type=int, default=12_778_496)
-    ap.add_argument("--ref-sample-elems", type=int, default=524_288)
+    ap.add_argument("--cpu-sample-elems", type=int, default=25_557_032)
+    ap.add_argument("--ref-sample-elems", type=int, default=4_194_304)
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
