@@ -58,7 +58,6 @@ extern "C" {
 #define QESGD_SCALE_FIXED 2u /* scale = s*delta with the grid spacing delta given  */
 
 #define QESGD_STATUS_NONFINITE 1u /* a bucket held NaN/Inf or its norm overflowed fp32 */
-#define QESGD_STATUS_TIMEOUT 2u   /* a bounded device-side wait gave up: outputs are invalid */
 
 #define QESGD_MAX_WORKERS 64u
 #define QESGD_MIN_BUCKET 64u

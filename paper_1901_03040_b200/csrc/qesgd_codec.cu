@@ -772,10 +772,12 @@ cudaError_t launch_encode_v(const EncodeArgs &a, uint32_t K, int sm_count, cudaS
     (void)sm_count;
     constexpr int V = QESGD_ENCODE_CHUNKS;
     constexpr uint32_t SMALL = QESGD_ENCODE_WARPS;        // warps of the usual CTA
+    // a bucket never leaves its CTA: as many warps as the bucket spans, no more
+    const uint32_t need = (1u << a.log2_bucket) / (uint32_t)(V * CHUNK);
+    if (need <= SMALL) return launch_encode_w<BITS, MODE, ANCHOR, VEC, SMALL>(a, K, stream);
+    if (need <= 2u) return launch_encode_w<BITS, MODE, ANCHOR, VEC, (SMALL > 2 ? SMALL : 2)>(a, K, stream);
+    if (need <= 4u) return launch_encode_w<BITS, MODE, ANCHOR, VEC, (SMALL > 4 ? SMALL : 4)>(a, K, stream);
     constexpr uint32_t LARGE = QESGD_MAX_BUCKET / (V * CHUNK);   // enough for the widest bucket
-    // a bucket never leaves its CTA
-    if ((1u << a.log2_bucket) <= SMALL * V * CHUNK)
-        return launch_encode_w<BITS, MODE, ANCHOR, VEC, SMALL>(a, K, stream);
     return launch_encode_w<BITS, MODE, ANCHOR, VEC, (LARGE > SMALL ? LARGE : SMALL)>(a, K, stream);
 }
 
