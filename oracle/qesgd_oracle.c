@@ -287,6 +287,33 @@ int qesgd_ref_decode_average_apply(float *param, uint64_t n, uint32_t K, const u
     return QREF_OK;
 }
 
+/* Gradient compression on the push side (Sec. 3: "users can compress gradients"; the QSGD
+ * baseline of Sec. 5 quantises gradients): the K streams hold quantised gradients and the
+ * server takes w <- w + alpha * (1/K) sum_k g_k with alpha = -learning rate (Eq. 2 with the
+ * minibatch mean replaced by the mean of the decoded workers).  alpha = 1 is the averaging
+ * line of Algorithm 3.  fp64 sum over k ascending, one rounding to fp32. */
+int qesgd_ref_decode_average_axpy(float *param, uint64_t n, uint32_t K, const uint32_t *codes,
+                                  uint64_t code_stride, const float *scales,
+                                  uint64_t scale_stride, uint32_t bucket, uint32_t s,
+                                  uint32_t bits, float alpha)
+{
+    if (!valid_bits(bits) || !valid_bucket(bucket) || K == 0) return QREF_EINVAL;
+    if (s < 1 || s > (1u << (bits - 1)) - 1u) return QREF_EINVAL;
+    if (n == 0) return QREF_OK;
+    if (!param || !codes || !scales) return QREF_EINVAL;
+    for (uint64_t e = 0; e < n; ++e) {
+        double sum = 0.0;
+        for (uint32_t k = 0; k < K; ++k) {
+            const uint32_t *ck = (const uint32_t *)((const char *)codes + (size_t)k * code_stride);
+            const float *sk = scales + (size_t)k * scale_stride;
+            float step = sk[e / bucket] / (float)s;
+            sum += (double)code_value(code_at(ck, e, bits), step, bits);
+        }
+        param[e] = (float)((double)param[e] + (double)alpha * (sum / (double)K));
+    }
+    return QREF_OK;
+}
+
 /* ------------------------------------------------------------------------ */
 /* Logistic regression (Sec. 1: f_i(w) = log(1 + exp(-y_i x_i^T w))) and the */
 /* minibatch SGD update of Eq. 2.  fp64 accumulation, u rounded to fp32 once */
@@ -342,5 +369,27 @@ int qesgd_ref_lr_local_epoch(const float *X, const float *y, uint64_t n_local, u
         int rc = qesgd_ref_lr_sgd_step(X + r * d, y + r, m, d, lr, u);
         if (rc != QREF_OK) return rc;
     }
+    return QREF_OK;
+}
+
+/* Minibatch mean gradient of the logistic loss at w (the summand of Eq. 2):
+ * g = (1/m) sum_j c_j x_j, c_j = -y_j / (1 + exp(y_j x_j^T w)); fp64, rounded once. */
+int qesgd_ref_lr_gradient(const float *Xb, const float *yb, uint32_t m, uint64_t d, const float *w,
+                          float *g)
+{
+    if (!Xb || !yb || !w || !g || m == 0 || d == 0) return QREF_EINVAL;
+    double *c = (double *)malloc(sizeof(double) * m);
+    if (!c) return QREF_ENOMEM;
+    for (uint32_t j = 0; j < m; ++j) {
+        double dot = 0.0;
+        for (uint64_t i = 0; i < d; ++i) dot += (double)Xb[(uint64_t)j * d + i] * (double)w[i];
+        c[j] = -(double)yb[j] / (1.0 + exp((double)yb[j] * dot));
+    }
+    for (uint64_t i = 0; i < d; ++i) {
+        double acc = 0.0;
+        for (uint32_t j = 0; j < m; ++j) acc += c[j] * (double)Xb[(uint64_t)j * d + i];
+        g[i] = (float)(acc / (double)m);
+    }
+    free(c);
     return QREF_OK;
 }

@@ -41,6 +41,11 @@ _lib.qesgd_ref_decode.restype = C.c_int
 _lib.qesgd_ref_decode_average_apply.argtypes = [_pf, _u64, _u32, _pu, _u64, _pf, _u64,
                                                 _u32, _u32, _u32]
 _lib.qesgd_ref_decode_average_apply.restype = C.c_int
+_lib.qesgd_ref_decode_average_axpy.argtypes = [_pf, _u64, _u32, _pu, _u64, _pf, _u64,
+                                               _u32, _u32, _u32, _f32]
+_lib.qesgd_ref_decode_average_axpy.restype = C.c_int
+_lib.qesgd_ref_lr_gradient.argtypes = [_pf, _pf, _u32, _u64, _pf, _pf]
+_lib.qesgd_ref_lr_gradient.restype = C.c_int
 _lib.qesgd_ref_lr_loss.argtypes = [_pf, _pf, _u64, _u64, _pf]
 _lib.qesgd_ref_lr_loss.restype = C.c_double
 _lib.qesgd_ref_lr_sgd_step.argtypes = [_pf, _pf, _u32, _u64, _f32, _pf]
@@ -135,6 +140,26 @@ def decode_average_apply(param, codes, scales, bucket, s, bits):
         _f(out), out.size, codes.shape[0], _u(codes), codes.shape[1] * 4, _f(scales),
         scales.shape[1], bucket, s, bits))
     return out
+
+
+def decode_average_axpy(param, codes, scales, bucket, s, bits, alpha):
+    """param + alpha * mean_k decode(stream k); codes uint32[K, words], scales float32[K, nb]."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint32)
+    scales = np.ascontiguousarray(scales, dtype=np.float32)
+    out = np.array(param, dtype=np.float32, copy=True)
+    _check(_lib.qesgd_ref_decode_average_axpy(
+        _f(out), out.size, codes.shape[0], _u(codes), codes.shape[1] * 4, _f(scales),
+        scales.shape[1], bucket, s, bits, alpha))
+    return out
+
+
+def lr_gradient(Xb, yb, w):
+    Xb = np.ascontiguousarray(Xb, dtype=np.float32)
+    g = np.zeros(Xb.shape[1], dtype=np.float32)
+    _check(_lib.qesgd_ref_lr_gradient(_f(Xb), _f(np.ascontiguousarray(yb, np.float32)),
+                                      Xb.shape[0], Xb.shape[1],
+                                      _f(np.ascontiguousarray(w, np.float32)), _f(g)))
+    return g
 
 
 def lr_loss(X, y, w):

@@ -496,6 +496,52 @@ def test_lr_step_from_zero_closed_form_and_epoch_descends():
     assert q.lr_loss(X, y2, u) < before - 0.05 and abs(before - math.log(2)) < 1e-12
 
 
+def test_lr_gradient_against_finite_differences_and_the_step():
+    m, d, lr = 9, 14, 0.3
+    X, y = _lr_data(m, d, 11)
+    w = (0.4 * np.random.default_rng(12).standard_normal(d)).astype(np.float32)
+    Xd, yd = X.astype(np.float64), y.astype(np.float64)
+
+    def loss(v):
+        return np.logaddexp(0.0, -yd * (Xd @ v)).mean()
+
+    fd = np.zeros(d)
+    eps = 1e-6
+    for i in range(d):
+        e = np.zeros(d)
+        e[i] = eps
+        fd[i] = (loss(w.astype(np.float64) + e) - loss(w.astype(np.float64) - e)) / (2 * eps)
+    g = q.lr_gradient(X, y, w)
+    assert np.abs(g - fd).max() < 2e-7
+    # Eq. 2: the step is w - lr * g
+    step = q.lr_sgd_step(X, y, lr, w)
+    assert np.abs(step - (w.astype(np.float64) - lr * g.astype(np.float64))).max() < 1e-7
+
+
+def test_average_axpy_is_linear_in_alpha_and_reduces_to_average_apply():
+    """w + alpha * mean_k g_k: alpha = 1 is the averaging line of Algorithm 3; alpha = -lr is the
+    SGD step of Eq. 2 on the mean of the decoded (quantised) gradients."""
+    rng = np.random.default_rng(21)
+    n, K, B, s, bits = 64 * 3 + 7, 4, 64, 7, 4
+    w = (0.05 * rng.standard_normal(n)).astype(np.float32)
+    codes, scales, dec = [], [], []
+    for k in range(K):
+        g = (1e-2 * rng.standard_normal(n)).astype(np.float32)
+        c, sc, _ = q.encode(g, None, B, s, bits, q.SCALE_NORM, 3, k, 0)
+        codes.append(c)
+        scales.append(sc)
+        dec.append(q.decode(c, sc, n, B, s, bits).astype(np.float64))
+    codes, scales = np.stack(codes), np.stack(scales)
+    mean = np.sum(dec, axis=0) / K
+    assert (q.decode_average_axpy(w, codes, scales, B, s, bits, 1.0)
+            == q.decode_average_apply(w, codes, scales, B, s, bits)).all()
+    for alpha in (-0.1, 0.5, -2.0):
+        got = q.decode_average_axpy(w, codes, scales, B, s, bits, alpha)
+        want = (w.astype(np.float64) + np.float64(np.float32(alpha)) * mean).astype(np.float32)
+        assert (got == want).all()
+    assert (q.decode_average_axpy(w, codes, scales, B, s, bits, 0.0) == w).all()
+
+
 def test_invalid_arguments_are_rejected():
     z = np.zeros(64, np.float32)
     for kw in (dict(bucket=48), dict(bucket=32), dict(bucket=16384), dict(bits=3),
