@@ -128,6 +128,20 @@ int qesgd_decode_average_apply(qesgd_ctx *ctx, float *param, uint64_t d, uint32_
                                const uint32_t *codes, uint64_t code_stride, const float *scales,
                                uint64_t scale_stride, uint32_t bucket, uint32_t s, uint32_t bits);
 
+/*
+ * Gradient compression on the push side (Sec. 3: "users can compress gradients"; the QSGD
+ * baseline of Sec. 5 quantises gradients with delta = ||g||): the K streams hold quantised
+ * gradients, encoded with anchor == NULL, and the server takes
+ *   param_i <- param_i + alpha * (1/K) * sum_k (+-level_{k,i} * fl32(scale_{k,bucket(i)} / s))
+ * with alpha = -learning rate (Eq. 2 on the mean of the decoded workers).  alpha = 1 is
+ * qesgd_decode_average_apply.  Same layout, limits and accuracy (1e-6 * max(|param_i|,
+ * |alpha| * max_k scale)); alpha must be finite.
+ */
+int qesgd_decode_average_axpy(qesgd_ctx *ctx, float *param, uint64_t d, uint32_t K,
+                              const uint32_t *codes, uint64_t code_stride, const float *scales,
+                              uint64_t scale_stride, uint32_t bucket, uint32_t s, uint32_t bits,
+                              float alpha);
+
 /* Decoding alone (the grid points delta*k of Eq. 3): out_i = +-level_i *
  * fl32(scale/s), i < d, bit-exact.  out: float[d]. */
 int qesgd_decode(qesgd_ctx *ctx, const uint32_t *codes, const float *scales, uint64_t d,
@@ -142,6 +156,11 @@ int qesgd_decode(qesgd_ctx *ctx, const uint32_t *codes, const float *scales, uin
  */
 int qesgd_lr_sgd_step(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32_t m, uint64_t d,
                       float lr, float *u);
+/* The summand of Eq. 2 alone: g_out = (1/m) * sum_j grad f_j(w) on the m rows of Xb, for
+ * workers that push (quantised) gradients instead of parameters.  w and g_out are float[d]
+ * and must not overlap.  Same two passes and accuracy as qesgd_lr_sgd_step. */
+int qesgd_lr_gradient(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32_t m, uint64_t d,
+                      const float *w, float *g_out);
 /* Rows [0, n_local) of X in consecutive minibatches of `batch` rows, in row
  * order; a last partial batch uses its own size in Eq. 2. */
 int qesgd_lr_local_epoch(qesgd_ctx *ctx, const float *X, const float *y, uint64_t n_local,

@@ -178,13 +178,15 @@ int qesgd_encode(qesgd_ctx *ctx, const float *local, const float *anchor, uint64
                               fixed_delta, seed, worker, epoch, codes_out, 0, scales_out, 0);
 }
 
-int qesgd_decode_average_apply(qesgd_ctx *ctx, float *param, uint64_t d, uint32_t K,
-                               const uint32_t *codes, uint64_t code_stride, const float *scales,
-                               uint64_t scale_stride, uint32_t bucket, uint32_t s, uint32_t bits)
+int qesgd_decode_average_axpy(qesgd_ctx *ctx, float *param, uint64_t d, uint32_t K,
+                              const uint32_t *codes, uint64_t code_stride, const float *scales,
+                              uint64_t scale_stride, uint32_t bucket, uint32_t s, uint32_t bits,
+                              float alpha)
 {
     if (!ctx) return QESGD_EINVAL;
     if (!valid_codec(bucket, s, bits)) return QESGD_EINVAL;
     if (K < 1 || K > QESGD_MAX_WORKERS) return QESGD_EINVAL;
+    if (!(alpha >= -3.402823466e38f && alpha <= 3.402823466e38f)) return QESGD_EINVAL;
     if (d == 0) return QESGD_OK;
     if (!param || !codes || !scales) return QESGD_EINVAL;
     if (!aligned(param, 4) || !aligned(codes, 16) || !aligned(scales, 16)) return QESGD_EINVAL;
@@ -198,6 +200,7 @@ int qesgd_decode_average_apply(qesgd_ctx *ctx, float *param, uint64_t d, uint32_
     a.d = d;
     a.nb = nb;
     a.K = K;
+    a.avg_scale = alpha / (float)K;
     a.log2_bucket = (uint32_t)log2_exact(bucket);
     a.s = s;
     a.codes = codes;
@@ -210,6 +213,14 @@ int qesgd_decode_average_apply(qesgd_ctx *ctx, float *param, uint64_t d, uint32_
     if (e != 0) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return QESGD_OK;
+}
+
+int qesgd_decode_average_apply(qesgd_ctx *ctx, float *param, uint64_t d, uint32_t K,
+                               const uint32_t *codes, uint64_t code_stride, const float *scales,
+                               uint64_t scale_stride, uint32_t bucket, uint32_t s, uint32_t bits)
+{
+    return qesgd_decode_average_axpy(ctx, param, d, K, codes, code_stride, scales, scale_stride,
+                                     bucket, s, bits, 1.0f);
 }
 
 int qesgd_decode(qesgd_ctx *ctx, const uint32_t *codes, const float *scales, uint64_t d,
@@ -225,6 +236,7 @@ int qesgd_decode(qesgd_ctx *ctx, const uint32_t *codes, const float *scales, uin
     a.d = d;
     a.nb = qesgd_num_buckets(d, bucket);
     a.K = 1;
+    a.avg_scale = 1.0f;
     a.log2_bucket = (uint32_t)log2_exact(bucket);
     a.s = s;
     a.codes = codes;
@@ -277,6 +289,24 @@ int qesgd_lr_sgd_step(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32_t
 {
     if (m < 1 || m > QESGD_MAX_LR_BATCH) return QESGD_EINVAL;
     return qesgd_lr_local_epoch_batch(ctx, Xb, yb, m, d, 1, m, lr, u, 0);
+}
+
+int qesgd_lr_gradient(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32_t m, uint64_t d,
+                      const float *w, float *g_out)
+{
+    if (!ctx) return QESGD_EINVAL;
+    if (m < 1 || m > QESGD_MAX_LR_BATCH) return QESGD_EINVAL;
+    if (d == 0) return QESGD_OK;
+    if (!Xb || !yb || !w || !g_out || w == g_out) return QESGD_EINVAL;
+    if (!aligned(Xb, 4) || !aligned(yb, 4) || !aligned(w, 4) || !aligned(g_out, 4)) return QESGD_EINVAL;
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
+    int launched = 0;
+    const int e = qesgd_launch_lr_gradient(Xb, yb, m, d, w, g_out, ctx->d_lr_work,
+                                           ctx->lr_work_floats, ctx->stream, &launched);
+    ctx->launches += (uint64_t)launched;
+    if (e != 0) return cuda_fail(ctx, e);
+    return QESGD_OK;
 }
 
 int qesgd_status(qesgd_ctx *ctx, uint32_t *flags_out)

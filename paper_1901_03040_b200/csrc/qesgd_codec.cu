@@ -732,7 +732,7 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
             cw[i][1] = nx[i][1];
         }
     }
-    const float inv_k = __fdiv_rn(1.0f, (float)a.K);
+    const float inv_k = a.avg_scale;   // alpha / K
 #pragma unroll
     for (int o = 0; o < OPL; ++o) {
 #pragma unroll

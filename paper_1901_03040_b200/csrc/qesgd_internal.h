@@ -45,6 +45,7 @@ struct DecodeArgs {
     uint64_t d;
     uint64_t nb;
     uint32_t K;
+    float avg_scale;        // alpha / K applied to the sum over workers (1/K for the plain average)
     uint32_t log2_bucket;
     uint32_t s;
     const uint32_t *codes;
@@ -64,3 +65,7 @@ int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float 
                          uint64_t y_worker_stride, uint32_t m, uint64_t d, uint32_t K, float lr,
                          float *u, uint64_t u_stride, float *work, uint64_t work_floats,
                          cudaStream_t stream, int *launched);
+// Minibatch mean gradient at w into g (same two passes; the second writes instead of updating).
+int qesgd_launch_lr_gradient(const float *Xb, const float *yb, uint32_t m, uint64_t d,
+                             const float *w, float *g, float *work, uint64_t work_floats,
+                             cudaStream_t stream, int *launched);

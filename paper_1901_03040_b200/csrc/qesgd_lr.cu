@@ -29,7 +29,9 @@ struct LrArgs {
     uint32_t m;
     uint64_t d;
     float rate;          // lr / m
-    float *u;
+    const float *u;      // point the margins are taken at
+    float *dst;          // accumulate != 0: dst += step (dst == u); else dst = gradient
+    uint32_t accumulate;
     uint64_t u_stride;
     float *work;
     uint32_t parts;      // P
@@ -126,7 +128,7 @@ __global__ void __launch_bounds__(UPD_THREADS) qesgd_lr_update_kernel(const LrAr
     const uint32_t k = blockIdx.y;
     const float *__restrict__ X = a.X + (uint64_t)k * a.x_stride;
     const float *__restrict__ y = a.y + (uint64_t)k * a.y_stride;
-    float *__restrict__ u = a.u + (uint64_t)k * a.u_stride;
+    float *__restrict__ u = a.dst + (uint64_t)k * a.u_stride;
     const float *__restrict__ work = a.work + (uint64_t)k * a.parts * a.m;
     for (uint32_t j = threadIdx.x; j < a.m; j += blockDim.x) {
         float margin = 0.0f;
@@ -172,32 +174,38 @@ __global__ void __launch_bounds__(UPD_THREADS) qesgd_lr_update_kernel(const LrAr
             t.x += v.x; t.y += v.y; t.z += v.z; t.w += v.w;
         }
         if (VEC && c + 4 <= a.d) {
-            float4 uu = *reinterpret_cast<float4 *>(u + c);
+            float4 uu = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (a.accumulate) uu = *reinterpret_cast<float4 *>(u + c);
             uu.x += t.x; uu.y += t.y; uu.z += t.z; uu.w += t.w;
             *reinterpret_cast<float4 *>(u + c) = uu;
         } else {
-            u[c] += t.x;
-            if (c + 1 < a.d) u[c + 1] += t.y;
-            if (c + 2 < a.d) u[c + 2] += t.z;
-            if (c + 3 < a.d) u[c + 3] += t.w;
+            const bool acc_mode = a.accumulate != 0u;
+            u[c] = (acc_mode ? u[c] : 0.0f) + t.x;
+            if (c + 1 < a.d) u[c + 1] = (acc_mode ? u[c + 1] : 0.0f) + t.y;
+            if (c + 2 < a.d) u[c + 2] = (acc_mode ? u[c + 2] : 0.0f) + t.z;
+            if (c + 3 < a.d) u[c + 3] = (acc_mode ? u[c + 3] : 0.0f) + t.w;
         }
     }
 }
 
 }  // namespace
 
-int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float *yb,
-                         uint64_t y_worker_stride, uint32_t m, uint64_t d, uint32_t K, float lr,
-                         float *u, uint64_t u_stride, float *work, uint64_t work_floats,
-                         cudaStream_t stream, int *launched)
+namespace {
+
+// Both passes for K workers.  rate multiplies y_j / (1 + exp(y_j m_j)): lr/m for the SGD
+// step (dst = u, accumulated), -1/m for the mean gradient (dst = g, overwritten).
+int launch_lr_passes(const float *Xb, uint64_t x_worker_stride, const float *yb,
+                     uint64_t y_worker_stride, uint32_t m, uint64_t d, uint32_t K, float rate,
+                     const float *u, float *dst, bool accumulate, uint64_t u_stride, float *work,
+                     uint64_t work_floats, cudaStream_t stream, int *launched)
 {
     *launched = 0;
     LrArgs a;
     a.X = Xb; a.x_stride = x_worker_stride;
     a.y = yb; a.y_stride = y_worker_stride;
     a.m = m; a.d = d;
-    a.rate = lr / (float)m;
-    a.u = u; a.u_stride = u_stride;
+    a.rate = rate;
+    a.u = u; a.dst = dst; a.accumulate = accumulate ? 1u : 0u; a.u_stride = u_stride;
     a.work = work;
     const uint64_t nseg = (d + SEG - 1) / SEG;
     uint64_t parts = work_floats / ((uint64_t)K * m);
@@ -207,7 +215,7 @@ int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float 
     a.parts = (uint32_t)parts;
     a.nseg = (uint32_t)nseg;
     const bool vec = (d % 4 == 0) && (x_worker_stride % 4 == 0) && (u_stride % 4 == 0) &&
-                     (((uintptr_t)Xb | (uintptr_t)u) % 16 == 0);
+                     (((uintptr_t)Xb | (uintptr_t)u | (uintptr_t)dst) % 16 == 0);
     dim3 g1((unsigned)parts, K), b1(256);
     if (vec) qesgd_lr_margin_kernel<true><<<g1, b1, 0, stream>>>(a);
     else qesgd_lr_margin_kernel<false><<<g1, b1, 0, stream>>>(a);
@@ -222,6 +230,25 @@ int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float 
     e = cudaGetLastError();
     if (e == cudaSuccess) *launched = 2;
     return (int)e;
+}
+
+}  // namespace
+
+int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float *yb,
+                         uint64_t y_worker_stride, uint32_t m, uint64_t d, uint32_t K, float lr,
+                         float *u, uint64_t u_stride, float *work, uint64_t work_floats,
+                         cudaStream_t stream, int *launched)
+{
+    return launch_lr_passes(Xb, x_worker_stride, yb, y_worker_stride, m, d, K, lr / (float)m, u, u,
+                            true, u_stride, work, work_floats, stream, launched);
+}
+
+int qesgd_launch_lr_gradient(const float *Xb, const float *yb, uint32_t m, uint64_t d,
+                             const float *w, float *g, float *work, uint64_t work_floats,
+                             cudaStream_t stream, int *launched)
+{
+    return launch_lr_passes(Xb, 0, yb, 0, m, d, 1, -1.0f / (float)m, w, g, false, 0, work,
+                            work_floats, stream, launched);
 }
 
 // ---------------------------------------------------------------------------

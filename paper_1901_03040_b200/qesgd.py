@@ -37,7 +37,10 @@ SIGNATURES = {
                                   _u64, _u32, _u32, _vp, _u64, _vp, _u64]),
     "qesgd_decode_average_apply": (_int, [_vp, _vp, _u64, _u32, _vp, _u64, _vp, _u64, _u32, _u32,
                                           _u32]),
+    "qesgd_decode_average_axpy": (_int, [_vp, _vp, _u64, _u32, _vp, _u64, _vp, _u64, _u32, _u32,
+                                         _u32, _f32]),
     "qesgd_decode": (_int, [_vp, _vp, _vp, _u64, _u32, _u32, _u32, _vp]),
+    "qesgd_lr_gradient": (_int, [_vp, _vp, _vp, _u32, _u64, _vp, _vp]),
     "qesgd_lr_sgd_step": (_int, [_vp, _vp, _vp, _u32, _u64, _f32, _vp]),
     "qesgd_lr_local_epoch": (_int, [_vp, _vp, _vp, _u64, _u64, _u32, _f32, _vp]),
     "qesgd_lr_local_epoch_batch": (_int, [_vp, _vp, _vp, _u64, _u64, _u32, _u32, _f32, _vp, _u64]),
@@ -129,6 +132,12 @@ class Context:
                                                    code_stride, _ptr(scales), scale_stride,
                                                    bucket, s, bits))
 
+    def qesgd_decode_average_axpy(self, param, d, K, codes, code_stride, scales, scale_stride,
+                                  bucket, s, bits, alpha):
+        self._check(lib.qesgd_decode_average_axpy(self._h, _ptr(param), d, K, _ptr(codes),
+                                                  code_stride, _ptr(scales), scale_stride,
+                                                  bucket, s, bits, alpha))
+
     def qesgd_decode(self, codes, scales, d, bucket, s, bits, out):
         self._check(lib.qesgd_decode(self._h, _ptr(codes), _ptr(scales), d, bucket, s, bits,
                                      _ptr(out)))
@@ -136,6 +145,9 @@ class Context:
     # -- local epoch ---------------------------------------------------------
     def qesgd_lr_sgd_step(self, Xb, yb, m, d, lr, u):
         self._check(lib.qesgd_lr_sgd_step(self._h, _ptr(Xb), _ptr(yb), m, d, lr, _ptr(u)))
+
+    def qesgd_lr_gradient(self, Xb, yb, m, d, w, g_out):
+        self._check(lib.qesgd_lr_gradient(self._h, _ptr(Xb), _ptr(yb), m, d, _ptr(w), _ptr(g_out)))
 
     def qesgd_lr_local_epoch(self, X, y, n_local, d, batch, lr, u):
         self._check(lib.qesgd_lr_local_epoch(self._h, _ptr(X), _ptr(y), n_local, d, batch, lr,

@@ -264,6 +264,50 @@ def test_lr_local_epoch_and_batch_match_oracle():
     assert (t1.cpu().numpy() == got[0]).all()
 
 
+# ------------------------------------------- gradient compression (push side) ---
+@pytest.mark.parametrize("alpha", [-0.1, 1.0, -3.5])
+@pytest.mark.parametrize("K,bucket,bits,s", [(4, 128, 4, 7), (16, 256, 2, 1), (3, 1024, 8, 127)])
+def test_decode_average_axpy_matches_oracle(K, bucket, bits, s, alpha):
+    n = 8192 + 777
+    w = synthetic.anchor_vector(n, seed=K)
+    codes, scales = [], []
+    for k in range(K):
+        g = synthetic.delta_vector(n, 1e-2, seed=50 + K, worker=k, outlier_prob=0.01)
+        c, sc, _ = ref.encode(g, None, bucket, s, bits, ref.SCALE_NORM, 9, k, 1)
+        codes.append(c)
+        scales.append(sc)
+    codes, scales = np.stack(codes), np.stack(scales)
+    nb = scales.shape[1]
+    nb_pad = (nb + 3) // 4 * 4
+    t_scales = torch.zeros((K, nb_pad), dtype=torch.float32, device="cuda")
+    t_scales[:, :nb] = G.dev(scales)
+    p = G.dev(w)
+    G.ctx().qesgd_decode_average_axpy(p, n, K, G.dev(codes), codes.shape[1] * 4, t_scales, nb_pad,
+                                      bucket, s, bits, alpha)
+    got = p.cpu().numpy()
+    want = ref.decode_average_axpy(w, codes, scales, bucket, s, bits, alpha)
+    smax = np.repeat(scales.max(axis=0), bucket)[:n]
+    tol = 1e-6 * np.maximum(np.abs(want), abs(alpha) * smax)
+    assert (np.abs(got.astype(np.float64) - want) <= tol).all()
+
+
+@pytest.mark.parametrize("m,d", [(64, 65536), (33, 1001), (256, 4096)])
+def test_lr_gradient_matches_oracle_and_quantised_gradient_step(m, d):
+    X, y, _ = synthetic.logistic_problem(m, d, seed=3 * m + d)
+    w = (0.3 * synthetic.normal_f32(d, 1.0, 8)).astype(np.float32)
+    tg = torch.full((d + 4,), 9.0, dtype=torch.float32, device="cuda")
+    G.ctx().qesgd_lr_gradient(G.dev(X), G.dev(y), m, d, G.dev(w), tg)
+    assert (tg[d:] == 9.0).all().item()
+    g = tg[:d].cpu().numpy()
+    want = ref.lr_gradient(X, y, w)
+    assert np.linalg.norm(g - want) <= 1e-5 * np.linalg.norm(want)
+    assert np.abs(g - want).max() <= 1e-5 * np.abs(want).max()
+    # the worker pushes the quantised gradient, the server applies -lr * Q(g): hand-off parity
+    codes, scales, st = G.gpu_encode(g, None, 256, 127, 8, ref.SCALE_NORM, 5, 0, 0)
+    wc, ws, _ = ref.encode(g, None, 256, 127, 8, ref.SCALE_NORM, 5, 0, 0)
+    assert st == 0 and (codes == wc).all() and (scales.view(np.uint32) == ws.view(np.uint32)).all()
+
+
 # ------------------------------------------------------ argument checking ----
 def test_invalid_arguments_return_einval_and_launch_nothing():
     c = G.ctx()
