@@ -287,6 +287,32 @@ int qesgd_ref_decode_average_apply(float *param, uint64_t n, uint32_t K, const u
     return QREF_OK;
 }
 
+/* One inner step of QESGD after the gradient update (Algorithm 2: z_{t,k+1} =
+ * Q(z^_{t,k+1}), u_{t,k+1} = w_t + z_{t,k+1}; server task of Algorithm 3: z <- Q(z), send z):
+ * on entry u holds w_t + z^ (the parameter after the SGD step); it is quantised against the
+ * anchor w_t exactly as qesgd_ref_encode does (the inner step index plays the role of the
+ * epoch in the draw counter), then u <- fl32(w_t + Q(z^)) and, if zsum is given,
+ * zsum <- fl32(zsum + Q(z^)) (the running sum of the epoch average, last line of
+ * Algorithms 2 and 3).  Q(z^) is the decoded value fl32(level * fl32(scale/s)) with its sign.
+ * codes_out / scales_out receive the stream that would be sent to the workers. */
+int qesgd_ref_requantize(float *u, const float *anchor, uint64_t n, uint64_t i0, uint32_t bucket,
+                         uint32_t s, uint32_t bits, uint32_t scale_mode, float fixed_delta,
+                         uint64_t seed, uint32_t worker, uint32_t step, float *zsum,
+                         uint32_t *codes_out, float *scales_out, uint32_t *status)
+{
+    if (!anchor) return QREF_EINVAL;
+    int rc = qesgd_ref_encode(u, anchor, n, i0, bucket, s, bits, scale_mode, fixed_delta, seed,
+                              worker, step, codes_out, scales_out, status);
+    if (rc != QREF_OK) return rc;
+    for (uint64_t e = 0; e < n; ++e) {
+        float delta = scales_out[e / bucket] / (float)s;
+        float v = code_value(code_at(codes_out, e, bits), delta, bits);
+        u[e] = anchor[e] + v;
+        if (zsum) zsum[e] = zsum[e] + v;
+    }
+    return QREF_OK;
+}
+
 /* Gradient compression on the push side (Sec. 3: "users can compress gradients"; the QSGD
  * baseline of Sec. 5 quantises gradients): the K streams hold quantised gradients and the
  * server takes w <- w + alpha * (1/K) sum_k g_k with alpha = -learning rate (Eq. 2 with the

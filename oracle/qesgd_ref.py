@@ -41,6 +41,9 @@ _lib.qesgd_ref_decode.restype = C.c_int
 _lib.qesgd_ref_decode_average_apply.argtypes = [_pf, _u64, _u32, _pu, _u64, _pf, _u64,
                                                 _u32, _u32, _u32]
 _lib.qesgd_ref_decode_average_apply.restype = C.c_int
+_lib.qesgd_ref_requantize.argtypes = [_pf, _pf, _u64, _u64, _u32, _u32, _u32, _u32, _f32, _u64,
+                                      _u32, _u32, _pf, _pu, _pf, _pu]
+_lib.qesgd_ref_requantize.restype = C.c_int
 _lib.qesgd_ref_decode_average_axpy.argtypes = [_pf, _u64, _u32, _pu, _u64, _pf, _u64,
                                                _u32, _u32, _u32, _f32]
 _lib.qesgd_ref_decode_average_axpy.restype = C.c_int
@@ -140,6 +143,24 @@ def decode_average_apply(param, codes, scales, bucket, s, bits):
         _f(out), out.size, codes.shape[0], _u(codes), codes.shape[1] * 4, _f(scales),
         scales.shape[1], bucket, s, bits))
     return out
+
+
+def requantize(u, anchor, bucket, s, bits, scale_mode, seed, worker, step, zsum=None,
+               i0=0, fixed_delta=0.0):
+    """Returns (u_new, zsum_new or None, codes, scales, status); inputs are not modified."""
+    u = np.array(u, dtype=np.float32, copy=True)
+    anchor = np.ascontiguousarray(anchor, dtype=np.float32)
+    n = u.size
+    nb = num_buckets(n, bucket)
+    codes = np.zeros(nb * bucket * bits // 32, dtype=np.uint32)
+    scales = np.zeros(nb, dtype=np.float32)
+    status = np.zeros(1, dtype=np.uint32)
+    z = None if zsum is None else np.array(zsum, dtype=np.float32, copy=True)
+    _check(_lib.qesgd_ref_requantize(_f(u), _f(anchor), n, i0, bucket, s, bits, scale_mode,
+                                     fixed_delta, seed, worker, step,
+                                     _f(z) if z is not None else None, _u(codes), _f(scales),
+                                     _u(status)))
+    return u, z, codes, scales, int(status[0])
 
 
 def decode_average_axpy(param, codes, scales, bucket, s, bits, alpha):

@@ -542,6 +542,61 @@ def test_average_axpy_is_linear_in_alpha_and_reduces_to_average_apply():
     assert (q.decode_average_axpy(w, codes, scales, B, s, bits, 0.0) == w).all()
 
 
+# ----------------------------------------- per-step QESGD (Algorithms 2 and 3) --
+def test_requantize_is_encode_decode_and_add():
+    rng = np.random.default_rng(31)
+    n, B, s, bits = 64 * 3 + 9, 64, 7, 4
+    w = (0.05 * rng.standard_normal(n)).astype(np.float32)
+    u = (w + 1e-3 * rng.standard_normal(n)).astype(np.float32)
+    zsum = (1e-3 * rng.standard_normal(n)).astype(np.float32)
+    u2, z2, codes, scales, st = q.requantize(u, w, B, s, bits, q.SCALE_NORM, 5, 0, 3, zsum=zsum)
+    c, sc, _ = q.encode(u, w, B, s, bits, q.SCALE_NORM, 5, 0, 3)
+    v = q.decode(c, sc, n, B, s, bits)
+    assert st == 0 and (codes == c).all() and (scales == sc).all()
+    assert (u2 == w + v).all() and (z2 == zsum + v).all()         # numpy fp32 adds
+    assert np.abs(u2 - u).max() < scales.max() / s                 # moved by less than one grid step
+    # a point already on the grid (and exactly representable after the add) stays put
+    k = rng.integers(-7, 8, 64)
+    k[0] = 7
+    wg = (rng.integers(-100, 100, 64) * 2.0 ** -8).astype(np.float32)
+    ug = (wg + k * 2.0 ** -8).astype(np.float32)
+    u3, _, _, _, _ = q.requantize(ug, wg, 64, 7, 4, q.SCALE_MAX, 1, 0, 0)
+    assert (u3 == ug).all()
+
+
+def test_qesgd_epoch_average_and_eight_bits_track_sgd():
+    """Algorithm 2 on a small logistic problem: w_{t+1} = (1/K_t) sum_{k<K_t} u_{t,k}
+    = w_t + (1/K_t) sum_k z_{t,k}; with 8 bits the epoch ends close to Epoch-SGD (Algorithm 1),
+    as the end of Sec. 4 says."""
+    m, d, Kt, lr = 16, 256, 12, 0.5
+    rng = np.random.default_rng(41)
+    X = (rng.standard_normal((m * Kt, d)) / np.sqrt(d)).astype(np.float32)
+    y = np.sign(X.astype(np.float64) @ rng.standard_normal(d)).astype(np.float32)
+    w = np.zeros(d, dtype=np.float32)
+    delta = 5e-4                                   # grid spacing; the range +-127 * delta is never left
+    u, u_sgd = w.copy(), w.copy()
+    zsum = np.zeros(d, dtype=np.float32)
+    iterates, iterates_sgd = [], []
+    for k in range(Kt):
+        iterates.append(u.astype(np.float64))
+        iterates_sgd.append(u_sgd.astype(np.float64))
+        rows = slice(k * m, (k + 1) * m)
+        u = q.lr_sgd_step(X[rows], y[rows], lr, u)
+        u_sgd = q.lr_sgd_step(X[rows], y[rows], lr, u_sgd)
+        acc = zsum if k + 1 < Kt else None         # z_{t,K_t} is not part of the average
+        u, znew, _, _, st = q.requantize(u, w, 256, 127, 8, q.SCALE_FIXED, 7, 0, k, zsum=acc,
+                                         fixed_delta=delta)
+        assert st == 0
+        if znew is not None:
+            zsum = znew
+    w_next = w.astype(np.float64) + zsum.astype(np.float64) / Kt
+    assert np.abs(w_next - np.mean(iterates, axis=0)).max() < 1e-6
+    w_sgd = np.mean(iterates_sgd, axis=0)
+    # quantisation noise per step is at most delta/2 per coordinate and does not accumulate
+    assert np.abs(w_next - w_sgd).max() < 4 * delta
+    assert abs(q.lr_loss(X, y, w_next.astype(np.float32)) - q.lr_loss(X, y, w_sgd.astype(np.float32))) < 1e-3
+
+
 def test_invalid_arguments_are_rejected():
     z = np.zeros(64, np.float32)
     for kw in (dict(bucket=48), dict(bucket=32), dict(bucket=16384), dict(bits=3),
