@@ -168,6 +168,8 @@ def run_ours(args):
         return run_c2(args, device, world, rank)
     if args.workload == "c1":
         return run_c1(args, device, world, rank)
+    if args.workload == "qstep":
+        return run_qstep(args, device, world, rank)
     w = dict(WORKLOADS[args.workload])
     if args.bucket:
         w["bucket"] = args.bucket
@@ -436,6 +438,56 @@ def run_c2(args, device, world, rank):
         print(json.dumps(line))
 
 
+def run_qstep(args, device, world, rank):
+    """Per-step QESGD (Algorithm 2): qesgd_requantize on one vector, d = 2^26 by default, 8-bit
+    codes with a caller-given grid spacing (the paper's own choice of delta), bucket 512, running
+    sum on.  Algorithmic bytes per element: u, anchor, zsum read (12) + u, zsum written (8) + code
+    (1) + scale (4/512)."""
+    import torch
+    from paper_1901_03040_b200 import qesgd, synthetic
+    d, B, s, bits = (args.d or (1 << 26)), 512, 127, 8
+    stream = torch.cuda.Stream(device)
+    ctx = qesgd.Context(device.index, stream)
+    w = synthetic.device_normal_f32((d,), synthetic.ANCHOR_SIGMA, 1, device)
+    u = w + synthetic.device_normal_f32((d,), 1e-3, 2, device)
+    zsum = torch.zeros(d, dtype=torch.float32, device=device)
+    codes, scales = qesgd.alloc_stream_buffers(1, d, B, bits, device)
+    mode = {"norm": qesgd.SCALE_NORM, "max": qesgd.SCALE_MAX, "fixed": qesgd.SCALE_FIXED}[args.scale_mode]
+
+    def call(i):
+        ctx.qesgd_requantize(u, w, d, B, s, bits, mode, 7, 0, i, zsum, codes, scales,
+                             fixed_delta=4e-3 / s)
+    for i in range(args.warmup):
+        call(i)
+    torch.cuda.synchronize()
+    launches0 = ctx.qesgd_launch_count()
+    sampler = ClockSampler(device.index) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        call(args.warmup + i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    clocks = sampler.stop() if sampler else None
+    ms = e0.elapsed_time(e1) / args.steps
+    nbytes = d * (12.0 + 8.0 + bits / 8.0 + 4.0 / B)
+    peak, peak_src = peaks()
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    line = {"metric": "requantize throughput, fp32-equivalent", "value": 4.0 * d / (ms * 1e-3) / 1e9,
+            "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "per-step QESGD: qesgd_requantize, 8-bit, bucket 512, running sum",
+                       "d": d, "scale_mode": args.scale_mode, "l2": "five streams of 4*d bytes, larger than L2"},
+            "gpu_launches": int(ctx.qesgd_launch_count() - launches0),
+            "roofline": {"bound": "hbm", "kernel": "qesgd_encode_kernel (requantize)", "achieved": gbs,
+                         "peak": peak, "unit": "GB/s", "frac": gbs / peak, "traffic": None,
+                         "peak_source": peak_src, "algorithmic_bytes_per_launch": nbytes},
+            "status_flags": ctx.qesgd_status(), "clocks": clocks}
+    if rank == 0:
+        print(json.dumps(line))
+
+
 def run_c1(args, device, world, rank):
     """End-to-end QESGD round on logistic regression: K=4 workers run one local epoch of
     minibatch-64 SGD from the anchor, encode (8-bit, bucket 512), server applies."""
@@ -555,7 +607,7 @@ def main():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["c4", "c3", "c5", "c2", "c1"], default="c4")
+    ap.add_argument("--workload", choices=["c4", "c3", "c5", "c2", "c1", "qstep"], default="c4")
     ap.add_argument("--bucket", type=int, default=0, help="override the bucket size (c5 sweep)")
     ap.add_argument("--d", type=int, default=0, help="vector length for --workload c2")
     ap.add_argument("--scale-mode", choices=["norm", "max", "fixed"], default="norm",

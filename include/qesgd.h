@@ -129,6 +129,24 @@ int qesgd_decode_average_apply(qesgd_ctx *ctx, float *param, uint64_t d, uint32_
                                uint64_t scale_stride, uint32_t bucket, uint32_t s, uint32_t bits);
 
 /*
+ * Per-step QESGD (Algorithm 2: z_{t,k+1} = Q(z^_{t,k+1}), u_{t,k+1} = w_t + z_{t,k+1};
+ * server task of Algorithm 3: z <- Q(z), send z to all workers).  On entry u (float[d])
+ * holds w_t + z^, the parameter after the gradient step.  In one pass the delta against
+ * `anchor` (= w_t, required) is quantised exactly as by qesgd_encode (`step`, the inner
+ * iteration index, takes the place of the epoch in the draw counter; the stream that would
+ * be sent goes to codes_out / scales_out), u is overwritten with fl32(anchor + Q(z^)), and,
+ * if zsum != NULL, zsum_i <- fl32(zsum_i + Q(z^)_i): the running sum of the epoch average
+ * w_{t+1} = w_t + (1/K_t) sum_k z_{t,k} (last line of Algorithms 2 and 3; apply it with any
+ * axpy).  Q(z^)_i = +-level_i * fl32(scale/s).  Everything is bit-exact against the oracle.
+ * u and zsum (float[d]) must both or neither be 32-byte aligned; other arguments as for
+ * qesgd_encode.
+ */
+int qesgd_requantize(qesgd_ctx *ctx, float *u, const float *anchor, uint64_t d, uint32_t bucket,
+                     uint32_t s, uint32_t bits, uint32_t scale_mode, float fixed_delta,
+                     uint64_t seed, uint32_t worker, uint32_t step, float *zsum,
+                     uint32_t *codes_out, float *scales_out);
+
+/*
  * Gradient compression on the push side (Sec. 3: "users can compress gradients"; the QSGD
  * baseline of Sec. 5 quantises gradients with delta = ||g||): the K streams hold quantised
  * gradients, encoded with anchor == NULL, and the server takes

@@ -118,11 +118,12 @@ uint64_t qesgd_code_bytes(uint64_t d, uint32_t bucket, uint32_t bits)
     return qesgd_num_buckets(d, bucket) * (bucket / 8u) * bits;
 }
 
-int qesgd_encode_batch(qesgd_ctx *ctx, const float *local, uint64_t local_stride,
+static int encode_impl(qesgd_ctx *ctx, const float *local, uint64_t local_stride,
                        const float *anchor, uint64_t d, uint32_t K, uint32_t bucket, uint32_t s,
                        uint32_t bits, uint32_t scale_mode, float fixed_delta, uint64_t seed,
                        uint32_t worker0, uint32_t epoch, uint32_t *codes_out,
-                       uint64_t code_stride, float *scales_out, uint64_t scale_stride)
+                       uint64_t code_stride, float *scales_out, uint64_t scale_stride,
+                       float *u_out, float *zsum)
 {
     if (!ctx) return QESGD_EINVAL;
     if (!valid_codec(bucket, s, bits) || scale_mode > QESGD_SCALE_FIXED) return QESGD_EINVAL;
@@ -160,6 +161,8 @@ int qesgd_encode_batch(qesgd_ctx *ctx, const float *local, uint64_t local_stride
     a.scales = scales_out;
     a.scale_stride = K > 1 ? scale_stride : 0;
     a.status = ctx->d_status;
+    a.u_out = u_out;
+    a.zsum = zsum;
     const bool vec = aligned(local, 32) && aligned(anchor, 32) && (a.local_stride % 8 == 0);
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
@@ -167,6 +170,29 @@ int qesgd_encode_batch(qesgd_ctx *ctx, const float *local, uint64_t local_stride
     if (e != 0) return cuda_fail(ctx, e);
     ctx->launches += 1;
     return QESGD_OK;
+}
+
+int qesgd_encode_batch(qesgd_ctx *ctx, const float *local, uint64_t local_stride,
+                       const float *anchor, uint64_t d, uint32_t K, uint32_t bucket, uint32_t s,
+                       uint32_t bits, uint32_t scale_mode, float fixed_delta, uint64_t seed,
+                       uint32_t worker0, uint32_t epoch, uint32_t *codes_out,
+                       uint64_t code_stride, float *scales_out, uint64_t scale_stride)
+{
+    return encode_impl(ctx, local, local_stride, anchor, d, K, bucket, s, bits, scale_mode,
+                       fixed_delta, seed, worker0, epoch, codes_out, code_stride, scales_out,
+                       scale_stride, nullptr, nullptr);
+}
+
+int qesgd_requantize(qesgd_ctx *ctx, float *u, const float *anchor, uint64_t d, uint32_t bucket,
+                     uint32_t s, uint32_t bits, uint32_t scale_mode, float fixed_delta,
+                     uint64_t seed, uint32_t worker, uint32_t step, float *zsum,
+                     uint32_t *codes_out, float *scales_out)
+{
+    if (!anchor || !u) return QESGD_EINVAL;
+    if (zsum && !aligned(zsum, 4)) return QESGD_EINVAL;
+    if (zsum && (aligned(u, 32) != aligned(zsum, 32))) return QESGD_EINVAL;  // one load path for both
+    return encode_impl(ctx, u, 0, anchor, d, 1, bucket, s, bits, scale_mode, fixed_delta, seed,
+                       worker, step, codes_out, 0, scales_out, 0, u, zsum);
 }
 
 int qesgd_encode(qesgd_ctx *ctx, const float *local, const float *anchor, uint64_t d,

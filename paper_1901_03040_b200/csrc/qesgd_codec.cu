@@ -61,15 +61,16 @@ __device__ __forceinline__ void st256(float *p, const float (&v)[8])
 }
 
 // 8 elements starting at element index eb of a vector of d elements; zeros past d.
-template <bool VEC>
-__device__ __forceinline__ void load_octet(const float *__restrict__ p, uint64_t eb, uint64_t d,
-                                           float (&v)[8])
+// RW = the buffer is also written by this kernel: no read-only (non-coherent) loads.
+template <bool VEC, bool RW = false>
+__device__ __forceinline__ void load_octet(const float *p, uint64_t eb, uint64_t d, float (&v)[8])
 {
     if (VEC && eb + 8 <= d) {
-        ld256(p + eb, v);
+        if (RW) ld256_rw(p + eb, v);
+        else ld256(p + eb, v);
     } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = (eb + j < d) ? __ldg(p + eb + j) : 0.0f;
+        for (int j = 0; j < 8; ++j) v[j] = (eb + j < d) ? (RW ? p[eb + j] : __ldg(p + eb + j)) : 0.0f;
     }
 }
 
@@ -324,7 +325,10 @@ struct EncodeShared {
 // Philox draws, stochastic rounding, packing, stores.  `iter` selects the half of the
 // cross-warp scratch (callers alternate it between consecutive tiles of one CTA).
 // FULL = the whole warp tile lies inside the vector: no store needs a bounds check.
-template <int BITS, int MODE, int V, bool FULL>
+// REQ = per-step QESGD (Algorithm 2: z = Q(z^), u = w_t + z): besides the stream, the
+// quantised delta is decoded on the spot, written back as u = fl32(anchor + Q(z)) and
+// added to the running sum of the epoch average.
+template <int BITS, int MODE, int V, bool FULL, bool REQ>
 __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)[V][8],
                                                  uint64_t warp_base, uint32_t k, uint32_t lane,
                                                  uint32_t warp, EncodeShared &sh, uint32_t iter)
@@ -332,7 +336,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
     constexpr uint32_t LOG2_WARP_ELEMS = V == 4 ? 10 : 9;
     const uint32_t lb = a.log2_bucket;
     const float sf = (float)a.s;
-    float my_scale, my_inv;
+    float my_scale, my_inv, my_delta = 0.0f;
     bool flag = false;
     // ---- per-bucket scale: one value per lane, then handed back per chunk ------
     if (MODE == 0) {
@@ -375,6 +379,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
         const bool ok = !nonfinite && my_scale >= 0x1p-100f;
         my_inv = ok ? __fdiv_rn(sf, my_scale) : 0.0f;
         my_scale = ok ? my_scale : 0.0f;
+        if (REQ) my_delta = __fdiv_rn(my_scale, sf);   // grid spacing of the decoder
         // Lanes past the padded length hold zeros, so a set flag always belongs to real data.
         flag = nonfinite;
     }
@@ -399,11 +404,12 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
     for (int c = 0; c < V; ++c) {
         const uint32_t off = (uint32_t)c * CHUNK + loff;        // element offset inside the tile
         const bool inside = FULL || warp_base + off < a.padded;
-        float scale = my_scale, inv = my_inv;
+        float scale = my_scale, inv = my_inv, delta = my_delta;
         if (MODE != 2) {   // fetch chunk c's bucket scale from the neighbour lane that carried it
             const int src = (int)lane_of_chunk<V>(lane, c);
             scale = __shfl_sync(FULL, my_scale, src);
             inv = __shfl_sync(FULL, my_inv, src);
+            if (REQ) delta = __shfl_sync(FULL, my_delta, src);
         }
         if (inside) {      // the first lane of every bucket writes its scale
             if (!wide) {
@@ -427,6 +433,43 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
             level_pair(z[c][j], z[c][j + 1], inv2, sf, x[j >> 1] & 0xFFFFu, x[j >> 1] >> 16,
                        X[j], X[j + 1]);
         }
+        if (REQ) {
+            // decode what was just quantised: +-level * delta, the sign only where level > 0
+            float v[8], w[8];
+            const uint64_t e0 = warp_base + off;
+            const uint64_t go = (uint64_t)k * a.local_stride + e0;
+            if (FULL) ld256(a.anchor + e0, w);
+            else load_octet<false>(a.anchor, e0, a.d, w);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const uint32_t lv = X[j] >> 16;
+                const float lf = __fsub_rn(__uint_as_float(0x4B000000u | lv), 8388608.0f);
+                const uint32_t sign31 = Z[j] & (lv + 0x7FFFFFFFu) & 0x80000000u;
+                v[j] = __uint_as_float(__float_as_uint(__fmul_rn(lf, delta)) | sign31);
+                w[j] = __fadd_rn(w[j], v[j]);
+            }
+            if (FULL) {
+                st256(a.u_out + go, w);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (e0 + j < a.d) a.u_out[go + j] = w[j];
+            }
+            if (a.zsum) {
+                float zs[8];
+                if (FULL) ld256_rw(a.zsum + go, zs);
+                else load_octet<false, true>(a.zsum, go, (uint64_t)k * a.local_stride + a.d, zs);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) zs[j] = __fadd_rn(zs[j], v[j]);
+                if (FULL) {
+                    st256(a.zsum + go, zs);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 8; ++j)
+                        if (e0 + j < a.d) a.zsum[go + j] = zs[j];
+                }
+            }
+        }
         uint32_t out[2];
         pack_octet<BITS>(X, Z, out);
         if (inside) {
@@ -446,7 +489,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
 // One CTA per (tile, worker); every lane requests all of its 256-bit loads before it
 // uses any of them, and several CTAs per SM overlap one another's load and arithmetic
 // phases.  VEC = false (pointers not 32-byte aligned) falls back to scalar loads.
-template <int BITS, int MODE, bool ANCHOR, bool VEC, int V, int WARPS>
+template <int BITS, int MODE, bool ANCHOR, bool VEC, int V, int WARPS, bool REQ>
 __global__ void __launch_bounds__(WARPS * 32, QESGD_ENCODE_MIN_WARPS / WARPS)
     qesgd_encode_kernel(const EncodeArgs a)
 {
@@ -464,7 +507,10 @@ __global__ void __launch_bounds__(WARPS * 32, QESGD_ENCODE_MIN_WARPS / WARPS)
     if (VEC && warp_base + V * CHUNK <= a.d) {   // the whole warp tile is inside the vector
         const float *__restrict__ p = local + warp_base + lane * 8u;
 #pragma unroll
-        for (int c = 0; c < V; ++c) ld256(p + c * CHUNK, z[c]);
+        for (int c = 0; c < V; ++c) {
+            if (REQ) ld256_rw(p + c * CHUNK, z[c]);   // u is written back below
+            else ld256(p + c * CHUNK, z[c]);
+        }
         if (ANCHOR) {
             const float *__restrict__ q = a.anchor + warp_base + lane * 8u;
             float w[V][8];
@@ -477,12 +523,12 @@ __global__ void __launch_bounds__(WARPS * 32, QESGD_ENCODE_MIN_WARPS / WARPS)
                     unpack2(sub2(pack2f(z[c][j], z[c][j + 1]), pack2f(w[c][j], w[c][j + 1])),
                             z[c][j], z[c][j + 1]);
         }
-        encode_warp_tile<BITS, MODE, V, true>(a, z, warp_base, k, lane, warp, sh, 0u);
+        encode_warp_tile<BITS, MODE, V, true, REQ>(a, z, warp_base, k, lane, warp, sh, 0u);
         return;
     }
 #pragma unroll
     for (int c = 0; c < V; ++c)
-        load_octet<VEC>(local, warp_base + (uint64_t)c * CHUNK + lane * 8u, a.d, z[c]);
+        load_octet<VEC, REQ>(local, warp_base + (uint64_t)c * CHUNK + lane * 8u, a.d, z[c]);
     if (ANCHOR) {
 #pragma unroll
         for (int c = 0; c < V; ++c) {
@@ -492,7 +538,7 @@ __global__ void __launch_bounds__(WARPS * 32, QESGD_ENCODE_MIN_WARPS / WARPS)
             for (int j = 0; j < 8; ++j) z[c][j] = __fsub_rn(z[c][j], w[j]);
         }
     }
-    encode_warp_tile<BITS, MODE, V, false>(a, z, warp_base, k, lane, warp, sh, 0u);
+    encode_warp_tile<BITS, MODE, V, false, REQ>(a, z, warp_base, k, lane, warp, sh, 0u);
 }
 
 // ------------------------------------------------------------- decode -------
@@ -762,7 +808,10 @@ cudaError_t launch_encode_w(const EncodeArgs &a, uint32_t K, cudaStream_t stream
     const uint64_t tiles = (a.padded + tile - 1) / tile;
     if (tiles == 0 || tiles * K > 0x7FFFFFFFull) return cudaErrorInvalidValue;
     dim3 grid((unsigned)(tiles * K), 1, 1), block(WARPS * 32u, 1, 1);
-    qesgd_encode_kernel<BITS, MODE, ANCHOR, VEC, V, WARPS><<<grid, block, 0, stream>>>(a);
+    if (ANCHOR && a.u_out)   // per-step QESGD: write back u = anchor + Q(z)
+        qesgd_encode_kernel<BITS, MODE, ANCHOR, VEC, V, WARPS, ANCHOR><<<grid, block, 0, stream>>>(a);
+    else
+        qesgd_encode_kernel<BITS, MODE, ANCHOR, VEC, V, WARPS, false><<<grid, block, 0, stream>>>(a);
     return cudaGetLastError();
 }
 

@@ -38,6 +38,8 @@ struct EncodeArgs {
     float *scales;
     uint64_t scale_stride;  // elements between workers
     uint32_t *status;
+    float *u_out;           // per-step QESGD: receives anchor + Q(z) (same layout as local); else null
+    float *zsum;            // per-step QESGD: running sum of Q(z), may be null
 };
 
 struct DecodeArgs {

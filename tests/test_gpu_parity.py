@@ -264,6 +264,78 @@ def test_lr_local_epoch_and_batch_match_oracle():
     assert (t1.cpu().numpy() == got[0]).all()
 
 
+# ----------------------------------------------- per-step QESGD (Algorithm 2) ---
+def _gpu_requantize(u, w, zsum, bucket, s, bits, mode, seed, worker, step, fixed_delta=0.0,
+                    misalign=0):
+    n = u.size
+    cb = qesgd.code_bytes(n, bucket, bits)
+    nb = qesgd.num_buckets(n, bucket)
+
+    def place(a):
+        buf = torch.full((n + misalign + 8,), 55.0, dtype=torch.float32, device="cuda")
+        buf[misalign:misalign + n] = G.dev(a)
+        return buf, buf[misalign:misalign + n]
+
+    bu, tu = place(u)
+    bz, tz = place(zsum) if zsum is not None else (None, None)
+    codes = torch.zeros(cb, dtype=torch.uint8, device="cuda")
+    scales = torch.zeros(nb + 3, dtype=torch.float32, device="cuda")
+    G.ctx().qesgd_requantize(tu, G.dev(w), n, bucket, s, bits, mode, seed, worker, step, tz, codes,
+                             scales, fixed_delta)
+    st = G.ctx().qesgd_status()
+    assert (bu[misalign + n:] == 55.0).all().item() and (bu[:misalign] == 55.0).all().item()
+    return (tu.cpu().numpy(), None if tz is None else tz.cpu().numpy(),
+            codes.cpu().numpy().view(np.uint32), scales[:nb].cpu().numpy(), st)
+
+
+@pytest.mark.parametrize("bucket", [64, 256, 1024, 4096])
+@pytest.mark.parametrize("bits,s,mode", [(8, 127, 2), (4, 7, 0), (2, 1, 1), (8, 100, 0)])
+def test_requantize_matches_oracle_bitwise(bits, s, mode, bucket):
+    n = 8192 * 2 + 1000 + 5
+    w = synthetic.anchor_vector(n, seed=bucket)
+    u = (w + synthetic.delta_vector(n, 1e-3, seed=bucket + 1, outlier_prob=0.01)).astype(np.float32)
+    zsum = synthetic.delta_vector(n, 1e-3, seed=bucket + 2)
+    delta = 3e-5
+    for misalign in (0, 3):
+        got = _gpu_requantize(u, w, zsum, bucket, s, bits, mode, 99, 1, 6, delta, misalign)
+        want = ref.requantize(u, w, bucket, s, bits, mode, 99, 1, 6, zsum=zsum, fixed_delta=delta)
+        assert (got[0].view(np.uint32) == want[0].view(np.uint32)).all()      # u
+        assert (got[1].view(np.uint32) == want[1].view(np.uint32)).all()      # running sum
+        assert (got[2] == want[2]).all()                                       # codes
+        assert (got[3].view(np.uint32) == want[3].view(np.uint32)).all()      # scales
+        assert got[4] == want[4]
+    got = _gpu_requantize(u, w, None, bucket, s, bits, mode, 99, 1, 6, delta)
+    want = ref.requantize(u, w, bucket, s, bits, mode, 99, 1, 6, fixed_delta=delta)
+    assert (got[0].view(np.uint32) == want[0].view(np.uint32)).all() and got[1] is None
+
+
+def test_qesgd_inner_loop_on_the_gpu_follows_the_oracle():
+    """Algorithm 2 on a logistic problem: gradient step, requantize, running sum; the GPU's
+    u after every step is handed to the oracle's requantize, which must agree bit for bit."""
+    m, d, Kt, lr, delta = 64, 4096, 6, 0.5, 2e-4
+    X, y, _ = synthetic.logistic_problem(m * Kt, d, seed=17)
+    tX, ty = G.dev(X), G.dev(y)
+    w = np.zeros(d, dtype=np.float32)
+    tw = G.dev(w)
+    tu = torch.zeros(d, dtype=torch.float32, device="cuda")
+    tz = torch.zeros(d, dtype=torch.float32, device="cuda")
+    codes = torch.zeros(qesgd.code_bytes(d, 512, 8), dtype=torch.uint8, device="cuda")
+    scales = torch.zeros(qesgd.num_buckets(d, 512), dtype=torch.float32, device="cuda")
+    c = G.ctx()
+    zsum_ref = np.zeros(d, dtype=np.float32)
+    for k in range(Kt):
+        rows = slice(k * m, (k + 1) * m)
+        c.qesgd_lr_sgd_step(tX[rows].contiguous(), ty[rows].contiguous(), m, d, lr, tu)
+        u_hat = tu.cpu().numpy()
+        c.qesgd_requantize(tu, tw, d, 512, 127, 8, qesgd.SCALE_FIXED, 3, 0, k, tz, codes, scales, delta)
+        u_ref, zsum_ref, c_ref, s_ref, _ = ref.requantize(u_hat, w, 512, 127, 8, ref.SCALE_FIXED, 3, 0, k,
+                                                          zsum=zsum_ref, fixed_delta=delta)
+        assert (tu.cpu().numpy().view(np.uint32) == u_ref.view(np.uint32)).all()
+        assert (tz.cpu().numpy().view(np.uint32) == zsum_ref.view(np.uint32)).all()
+        assert (codes.cpu().numpy().view(np.uint32) == c_ref).all()
+    assert c.qesgd_status() == 0 and np.abs(zsum_ref).max() > 0
+
+
 # ------------------------------------------- gradient compression (push side) ---
 @pytest.mark.parametrize("alpha", [-0.1, 1.0, -3.5])
 @pytest.mark.parametrize("K,bucket,bits,s", [(4, 128, 4, 7), (16, 256, 2, 1), (3, 1024, 8, 127)])
