@@ -78,23 +78,26 @@ __device__ __forceinline__ void load_octet(const float *p, uint64_t eb, uint64_t
 // Philox4x32 with 10 rounds (Salmon, Moraes, Dror, Shaw, SC'11), written from the
 // published round function: two 32x32->64 multiplies, the high halves xor'ed with
 // the other counter words and the round key; the key grows by the Weyl constants.
-__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                              const uint32_t (&rk)[10][2], uint32_t (&x)[4])
+// Two independent blocks advanced round by round: four multiply chains in flight instead
+// of two (measured 2 % faster than one block at a time; four at a time costs registers).
+// rk[r] = key + r * (0x9E3779B9, 0xBB67AE85): the ten round keys, prepared on the host so
+// that they reach the xor as kernel-parameter operands instead of per-thread additions.
+__device__ __forceinline__ void philox4x32_10_x2(uint32_t (&c)[2][4], const uint32_t (&rk)[10][2])
 {
-    // rk[r] = key + r * (0x9E3779B9, 0xBB67AE85): the ten round keys, prepared on the host so
-    // that they reach the xor as kernel-parameter operands instead of per-thread additions
 #pragma unroll
     for (int r = 0; r < 10; ++r) {
-        const uint64_t p0 = (uint64_t)0xD2511F53u * c0;
-        const uint64_t p1 = (uint64_t)0xCD9E8D57u * c2;
-        const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk[r][0];
-        const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk[r][1];
-        c1 = (uint32_t)p1;
-        c3 = (uint32_t)p0;
-        c0 = n0;
-        c2 = n2;
+#pragma unroll
+        for (int n = 0; n < 2; ++n) {
+            const uint64_t p0 = (uint64_t)0xD2511F53u * c[n][0];
+            const uint64_t p1 = (uint64_t)0xCD9E8D57u * c[n][2];
+            const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c[n][1] ^ rk[r][0];
+            const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c[n][3] ^ rk[r][1];
+            c[n][1] = (uint32_t)p1;
+            c[n][3] = (uint32_t)p0;
+            c[n][0] = n0;
+            c[n][2] = n2;
+        }
     }
-    x[0] = c0; x[1] = c1; x[2] = c2; x[3] = c3;
 }
 
 // ------------------------------------------------- packed fp32 pairs --------
@@ -399,6 +402,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
     const bool wide = lb > LOG2_WARP_ELEMS;                     // bucket spans several warps
     const bool wide_first = ((uint32_t)warp_base & bucket_mask) == 0u;   // this warp starts it
     const uint32_t wid = a.worker0 + k;
+    uint32_t xx[2][4];
 
 #pragma unroll
     for (int c = 0; c < V; ++c) {
@@ -419,8 +423,17 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
             }
         }
 
-        uint32_t x[4];
-        philox4x32_10(blk_lo + 32u * c, blk_hi, wid, a.epoch, a.round_key, x);
+        if ((c & 1) == 0) {   // draws for this chunk and the next, interleaved
+#pragma unroll
+            for (int n = 0; n < 2; ++n) {
+                xx[n][0] = blk_lo + 32u * (c + n);
+                xx[n][1] = blk_hi;
+                xx[n][2] = wid;
+                xx[n][3] = a.epoch;
+            }
+            philox4x32_10_x2(xx, a.round_key);
+        }
+        const uint32_t (&x)[4] = xx[c & 1];
 
         uint32_t X[8], Z[8];
         const uint64_t inv2 = pack2f(inv, inv);
