@@ -16,11 +16,14 @@ LIB = os.path.join(HERE, "libqesgd.so")
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 COMMON = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"),
           "-I", CSRC]
-UNITS = {
-    "qesgd_codec.cu": ["-fmad=false"],
-    "qesgd_lr.cu": [],
-    "qesgd_api.cu": [],
-}
+# (source, object name, extra flags): the codec is built once per code width, in parallel
+UNITS = [
+    ("qesgd_codec.cu", "qesgd_codec_2.o", ["-fmad=false", "-DQESGD_BITS=2"]),
+    ("qesgd_codec.cu", "qesgd_codec_4.o", ["-fmad=false", "-DQESGD_BITS=4"]),
+    ("qesgd_codec.cu", "qesgd_codec_8.o", ["-fmad=false", "-DQESGD_BITS=8"]),
+    ("qesgd_lr.cu", "qesgd_lr.o", []),
+    ("qesgd_api.cu", "qesgd_api.o", []),
+]
 
 
 def _nvcc():
@@ -44,9 +47,9 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = _nvcc()
     objs = []
     procs = []
-    for name, extra in UNITS.items():
+    for name, objname, extra in UNITS:
         src = os.path.join(CSRC, name)
-        obj = os.path.join(OBJ, name.replace(".cu", ".o"))
+        obj = os.path.join(OBJ, objname)
         objs.append(obj)
         if force or _stale(obj, [src] + headers):
             cmd = [nvcc] + ARCH + COMMON + extra + (["-Xptxas", "-v"] if verbose else []) + ["-c", src, "-o", obj]

@@ -867,47 +867,41 @@ cudaError_t launch_encode_b(const EncodeArgs &a, uint32_t K, uint32_t mode, bool
 
 }  // namespace
 
-int qesgd_launch_encode(const EncodeArgs &a, uint32_t K, uint32_t bits, uint32_t scale_mode,
-                        bool vec, int sm_count, cudaStream_t stream)
+// This file is compiled once per code width (-DQESGD_BITS=2, 4, 8) so that the three sets
+// of kernel instantiations build in parallel; qesgd_api.cu picks the set at run time.
+#ifndef QESGD_BITS
+#error "compile with -DQESGD_BITS=2, 4 or 8"
+#endif
+#define QESGD_CAT2(a, b) a##b
+#define QESGD_CAT(a, b) QESGD_CAT2(a, b)
+
+int QESGD_CAT(qesgd_launch_encode_, QESGD_BITS)(const EncodeArgs &a, uint32_t K, uint32_t scale_mode,
+                                                bool vec, int sm_count, cudaStream_t stream)
 {
-    switch (bits) {
-        case 2: return (int)launch_encode_b<2>(a, K, scale_mode, vec, sm_count, stream);
-        case 4: return (int)launch_encode_b<4>(a, K, scale_mode, vec, sm_count, stream);
-        default: return (int)launch_encode_b<8>(a, K, scale_mode, vec, sm_count, stream);
-    }
+    return (int)launch_encode_b<QESGD_BITS>(a, K, scale_mode, vec, sm_count, stream);
 }
 
-int qesgd_launch_decode(const DecodeArgs &a, uint32_t bits, bool vec, cudaStream_t stream)
+int QESGD_CAT(qesgd_launch_decode_, QESGD_BITS)(const DecodeArgs &a, bool vec, cudaStream_t stream)
 {
     const uint64_t octets = (a.d + 7) / 8;
     const uint64_t blocks = (octets + 255) / 256;
     if (blocks == 0 || blocks > 0x7FFFFFFFull) return (int)cudaErrorInvalidValue;
     dim3 grid((unsigned)blocks), block(256);
-#define QESGD_DEC(B)                                                                 \
-    if (vec) qesgd_decode_kernel<B, true><<<grid, block, 0, stream>>>(a);            \
-    else qesgd_decode_kernel<B, false><<<grid, block, 0, stream>>>(a)
-    if (bits == 2) { QESGD_DEC(2); }
-    else if (bits == 4) { QESGD_DEC(4); }
-    else { QESGD_DEC(8); }
-#undef QESGD_DEC
+    if (vec) qesgd_decode_kernel<QESGD_BITS, true><<<grid, block, 0, stream>>>(a);
+    else qesgd_decode_kernel<QESGD_BITS, false><<<grid, block, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }
 
-int qesgd_launch_decode_average_apply(const DecodeArgs &a, uint32_t bits, bool vec,
-                                      cudaStream_t stream)
+int QESGD_CAT(qesgd_launch_decode_average_apply_, QESGD_BITS)(const DecodeArgs &a, bool vec,
+                                                              cudaStream_t stream)
 {
-    const uint64_t warp_elems = 256ull * (8u / bits);   // one warp each (see the kernel)
+    const uint64_t warp_elems = 256ull * (8u / QESGD_BITS);   // one warp each (see the kernel)
     const uint64_t warps = (a.d + warp_elems - 1) / warp_elems;
     const uint64_t wpc = QESGD_DAA_THREADS / 32;
     const uint64_t blocks = (warps + wpc - 1) / wpc;
     if (blocks == 0 || blocks > 0x7FFFFFFFull) return (int)cudaErrorInvalidValue;
     dim3 grid((unsigned)blocks), block(QESGD_DAA_THREADS);
-#define QESGD_DAA(B)                                                                          \
-    if (vec) qesgd_decode_average_apply_kernel<B, true><<<grid, block, 0, stream>>>(a);       \
-    else qesgd_decode_average_apply_kernel<B, false><<<grid, block, 0, stream>>>(a)
-    if (bits == 2) { QESGD_DAA(2); }
-    else if (bits == 4) { QESGD_DAA(4); }
-    else { QESGD_DAA(8); }
-#undef QESGD_DAA
+    if (vec) qesgd_decode_average_apply_kernel<QESGD_BITS, true><<<grid, block, 0, stream>>>(a);
+    else qesgd_decode_average_apply_kernel<QESGD_BITS, false><<<grid, block, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }

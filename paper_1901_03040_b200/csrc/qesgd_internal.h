@@ -56,12 +56,44 @@ struct DecodeArgs {
     uint64_t scale_stride;  // elements
 };
 
-// Launchers (defined in qesgd_codec.cu / qesgd_lr.cu).  Return a cudaError_t as int.
-int qesgd_launch_encode(const EncodeArgs &a, uint32_t K, uint32_t bits, uint32_t scale_mode,
-                        bool vec, int sm_count, cudaStream_t stream);
-int qesgd_launch_decode(const DecodeArgs &a, uint32_t bits, bool vec, cudaStream_t stream);
-int qesgd_launch_decode_average_apply(const DecodeArgs &a, uint32_t bits, bool vec,
-                                      cudaStream_t stream);
+// Launchers.  Return a cudaError_t as int.  qesgd_codec.cu is compiled once per code width
+// and defines the *_2, *_4, *_8 functions; the width-dispatching wrappers are inline here.
+#define QESGD_DECLARE_WIDTH(B)                                                                  \
+    int qesgd_launch_encode_##B(const EncodeArgs &a, uint32_t K, uint32_t scale_mode, bool vec, \
+                                int sm_count, cudaStream_t stream);                             \
+    int qesgd_launch_decode_##B(const DecodeArgs &a, bool vec, cudaStream_t stream);            \
+    int qesgd_launch_decode_average_apply_##B(const DecodeArgs &a, bool vec, cudaStream_t stream);
+QESGD_DECLARE_WIDTH(2)
+QESGD_DECLARE_WIDTH(4)
+QESGD_DECLARE_WIDTH(8)
+#undef QESGD_DECLARE_WIDTH
+
+inline int qesgd_launch_encode(const EncodeArgs &a, uint32_t K, uint32_t bits, uint32_t scale_mode,
+                               bool vec, int sm_count, cudaStream_t stream)
+{
+    switch (bits) {
+        case 2: return qesgd_launch_encode_2(a, K, scale_mode, vec, sm_count, stream);
+        case 4: return qesgd_launch_encode_4(a, K, scale_mode, vec, sm_count, stream);
+        default: return qesgd_launch_encode_8(a, K, scale_mode, vec, sm_count, stream);
+    }
+}
+inline int qesgd_launch_decode(const DecodeArgs &a, uint32_t bits, bool vec, cudaStream_t stream)
+{
+    switch (bits) {
+        case 2: return qesgd_launch_decode_2(a, vec, stream);
+        case 4: return qesgd_launch_decode_4(a, vec, stream);
+        default: return qesgd_launch_decode_8(a, vec, stream);
+    }
+}
+inline int qesgd_launch_decode_average_apply(const DecodeArgs &a, uint32_t bits, bool vec,
+                                             cudaStream_t stream)
+{
+    switch (bits) {
+        case 2: return qesgd_launch_decode_average_apply_2(a, vec, stream);
+        case 4: return qesgd_launch_decode_average_apply_4(a, vec, stream);
+        default: return qesgd_launch_decode_average_apply_8(a, vec, stream);
+    }
+}
 // One minibatch step for K workers; returns the number of kernels launched in *launched.
 int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float *yb,
                          uint64_t y_worker_stride, uint32_t m, uint64_t d, uint32_t K, float lr,
