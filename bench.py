@@ -197,28 +197,45 @@ def run_ours(args):
     for i in range(args.warmup):
         step(i)
     barrier()
-    launches0 = ctx.qesgd_launch_count()
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    sampler = ClockSampler(local) if rank == 0 else None
-    t_begin = torch.cuda.Event(enable_timing=True)
-    t_end = torch.cuda.Event(enable_timing=True)
-    t_begin.record(stream)
-    for i in range(args.steps):
-        ev[i][0].record(stream)
-        ctx.qesgd_encode_batch(locs, stride, param, d, K, B, s, bits, qesgd.SCALE_NORM, 2024, 0,
-                               args.warmup + i, codes, codes.stride(0), scales, scales.stride(0))
-        ev[i][1].record(stream)
-        ctx.qesgd_decode_average_apply(param, d, K, codes, codes.stride(0), scales,
-                                       scales.stride(0), B, s, bits)
-        ev[i][2].record(stream)
-    t_end.record(stream)
-    barrier()
-    clocks = sampler.stop() if sampler else None
-    launches = ctx.qesgd_launch_count() - launches0
+    def timed_region(first_epoch):
+        launches0 = ctx.qesgd_launch_count()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+        sampler = ClockSampler(local) if rank == 0 else None
+        t_begin = torch.cuda.Event(enable_timing=True)
+        t_end = torch.cuda.Event(enable_timing=True)
+        t_begin.record(stream)
+        for i in range(args.steps):
+            ev[i][0].record(stream)
+            ctx.qesgd_encode_batch(locs, stride, param, d, K, B, s, bits, qesgd.SCALE_NORM, 2024, 0,
+                                   first_epoch + i, codes, codes.stride(0), scales, scales.stride(0))
+            ev[i][1].record(stream)
+            ctx.qesgd_decode_average_apply(param, d, K, codes, codes.stride(0), scales,
+                                           scales.stride(0), B, s, bits)
+            ev[i][2].record(stream)
+        t_end.record(stream)
+        barrier()
+        clk = sampler.stop() if sampler else None
+        return (t_begin.elapsed_time(t_end), [e[0].elapsed_time(e[1]) for e in ev],
+                [e[1].elapsed_time(e[2]) for e in ev], clk, ctx.qesgd_launch_count() - launches0)
+
+    def clocks_bad(clk):
+        if not clk:
+            return False
+        bad = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"} & set(clk["reasons"])
+        stuck = not clk["reasons"] and clk["sm_mhz"] < 0.6 * clk["sm_max_mhz"]
+        return bool(bad) or stuck
+
+    total_ms, enc_ms, daa_ms, clocks, launches = timed_region(args.warmup)
+    remeasured = False
+    again = 1.0 if (rank == 0 and clocks_bad(clocks)) else 0.0
+    _, again = aggregate_over_ranks(0.0, again, world, device, world > 1)
+    if again > 0.0:       # thermal or hardware slowdown, or clocks pinned low: measure once more
+        remeasured = True
+        total_ms, enc_ms, daa_ms, clocks, launches = timed_region(args.warmup + args.steps)
+    if clocks is not None:
+        clocks["remeasured"] = remeasured
+        clocks["rejected"] = clocks_bad(clocks)
     status = ctx.qesgd_status()
-    total_ms = t_begin.elapsed_time(t_end)
-    enc_ms = [e[0].elapsed_time(e[1]) for e in ev]
-    daa_ms = [e[1].elapsed_time(e[2]) for e in ev]
 
     fp32_equiv_bytes = 2.0 * 4.0 * d * K * args.steps
     ms_all, units_all = aggregate_over_ranks(total_ms, fp32_equiv_bytes, world, device, world > 1)
