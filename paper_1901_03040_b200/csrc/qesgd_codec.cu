@@ -341,6 +341,33 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
     const float sf = (float)a.s;
     float my_scale, my_inv, my_delta = 0.0f;
     bool flag = false;
+    // All addresses of the tile derive from three values computed once; inside the
+    // chunk loop only small compile-time offsets are added.  warp_base is a multiple of
+    // V*256, so the Philox block index (warp_base/8 + lane + 32c) never carries into
+    // its high word when c advances.
+    const uint32_t loff = lane * 8u;
+    uint8_t *const cbase = reinterpret_cast<uint8_t *>(a.codes) + (uint64_t)k * a.code_stride +
+                           ((warp_base + loff) >> 3) * (uint64_t)BITS;
+    float *const sbase = a.scales + (uint64_t)k * a.scale_stride + (warp_base >> lb);
+    const uint64_t blk0 = (warp_base >> 3) + lane;
+    const uint32_t blk_lo = (uint32_t)blk0, blk_hi = (uint32_t)(blk0 >> 32);
+    const uint32_t bucket_mask = (1u << lb) - 1u;
+    const bool wide = lb > LOG2_WARP_ELEMS;                     // bucket spans several warps
+    const bool wide_first = ((uint32_t)warp_base & bucket_mask) == 0u;   // this warp starts it
+    const uint32_t wid = a.worker0 + k;
+    uint32_t xx[2][4];
+
+    // The draws of the first two chunks are computed before the scale: they depend on nothing
+    // loaded, so they fill the time the reduction's shuffles and the square root wait.
+#pragma unroll
+    for (int n = 0; n < 2; ++n) {
+        xx[n][0] = blk_lo + 32u * n;
+        xx[n][1] = blk_hi;
+        xx[n][2] = wid;
+        xx[n][3] = a.epoch;
+    }
+    philox4x32_10_x2(xx, a.round_key);
+
     // ---- per-bucket scale: one value per lane, then handed back per chunk ------
     if (MODE == 0) {
         // fp64 sum of squares over the balanced binary tree on index order.  The product
@@ -388,22 +415,6 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
     }
 
     // ---- rounding, packing, stores ---------------------------------------------
-    // All addresses of the tile derive from three values computed once; inside the
-    // chunk loop only small compile-time offsets are added.  warp_base is a multiple of
-    // V*256, so the Philox block index (warp_base/8 + lane + 32c) never carries into
-    // its high word when c advances.
-    const uint32_t loff = lane * 8u;
-    uint8_t *const cbase = reinterpret_cast<uint8_t *>(a.codes) + (uint64_t)k * a.code_stride +
-                           ((warp_base + loff) >> 3) * (uint64_t)BITS;
-    float *const sbase = a.scales + (uint64_t)k * a.scale_stride + (warp_base >> lb);
-    const uint64_t blk0 = (warp_base >> 3) + lane;
-    const uint32_t blk_lo = (uint32_t)blk0, blk_hi = (uint32_t)(blk0 >> 32);
-    const uint32_t bucket_mask = (1u << lb) - 1u;
-    const bool wide = lb > LOG2_WARP_ELEMS;                     // bucket spans several warps
-    const bool wide_first = ((uint32_t)warp_base & bucket_mask) == 0u;   // this warp starts it
-    const uint32_t wid = a.worker0 + k;
-    uint32_t xx[2][4];
-
 #pragma unroll
     for (int c = 0; c < V; ++c) {
         const uint32_t off = (uint32_t)c * CHUNK + loff;        // element offset inside the tile
@@ -423,7 +434,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
             }
         }
 
-        if ((c & 1) == 0) {   // draws for this chunk and the next, interleaved
+        if ((c & 1) == 0 && c > 0) {   // draws for this chunk and the next, interleaved
 #pragma unroll
             for (int n = 0; n < 2; ++n) {
                 xx[n][0] = blk_lo + 32u * (c + n);
