@@ -155,9 +155,20 @@ def run_ours(args):
     import numpy as np
     import torch
     import torch.distributed as dist
-    from paper_1901_03040_b200 import qesgd
 
     world, rank, local = dist_info()
+    # build in-tree if the sources are newer (no-op otherwise); there is no fallback path
+    from paper_1901_03040_b200 import build as lib_build
+    if rank == 0:
+        lib_build.build()
+    else:           # other ranks wait for rank 0's build instead of racing it
+        sources = [os.path.join(lib_build.CSRC, f) for f in os.listdir(lib_build.CSRC)]
+        for _ in range(360):
+            if os.path.exists(lib_build.LIB) and not lib_build._stale(lib_build.LIB, sources):
+                break
+            time.sleep(0.5)
+    from paper_1901_03040_b200 import qesgd
+
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device; the CUDA path has no fallback")
     torch.cuda.set_device(local)
