@@ -85,6 +85,28 @@ def test_encode_batch_uses_worker_ids_and_strides():
         assert (gc[k] == wc).all() and (gs[k].view(np.uint32) == ws.view(np.uint32)).all()
 
 
+def test_encode_batch_with_the_largest_worker_count_and_padded_strides():
+    K, n, bucket, bits, s = 64, 2048 + 24, 64, 2, 1
+    w = synthetic.anchor_vector(n, seed=3)
+    locs = synthetic.worker_locals(w, K, 1e-4, seed=4)
+    c = G.ctx()
+    stride = n + 40                                          # more than the minimum, multiple of 8
+    buf = torch.zeros((K, stride), dtype=torch.float32, device="cuda")
+    buf[:, :n] = G.dev(locs)
+    cb, nb = qesgd.code_bytes(n, bucket, bits), qesgd.num_buckets(n, bucket)
+    codes = torch.full((K, cb + 32), 0xCD, dtype=torch.uint8, device="cuda")
+    scales = torch.full((K, nb + 7 + (4 - (nb + 7) % 4) % 4), -1.0, dtype=torch.float32, device="cuda")
+    c.qesgd_encode_batch(buf, stride, G.dev(w), n, K, bucket, s, bits, ref.SCALE_MAX, 8, 100, 2,
+                         codes, codes.stride(0), scales, scales.stride(0))
+    assert c.qesgd_status() == 0
+    assert (codes[:, cb:] == 0xCD).all().item() and (scales[:, nb:] == -1.0).all().item()
+    gc = codes[:, :cb].contiguous().cpu().numpy().view(np.uint32)
+    gs = scales[:, :nb].cpu().numpy()
+    for k in (0, 1, 31, 63):
+        wc, ws, _ = ref.encode(locs[k], w, bucket, s, bits, ref.SCALE_MAX, 8, 100 + k, 2)
+        assert (gc[k] == wc).all() and (gs[k].view(np.uint32) == ws.view(np.uint32)).all()
+
+
 def test_encode_epoch_and_seed_change_the_draws_but_not_the_scales():
     z = _delta(4096, seed=8)
     a = G.gpu_encode(z, None, 512, 7, 4, ref.SCALE_NORM, 1, 0, 0)
