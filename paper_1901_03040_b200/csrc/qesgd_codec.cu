@@ -25,7 +25,7 @@ constexpr int CHUNK = 256;  // elements covered by one warp-wide 256-bit load
 #define QESGD_DAA_BATCH 4       // workers whose code words are fetched together
 #endif
 #ifndef QESGD_DAA_MIN_CTAS
-#define QESGD_DAA_MIN_CTAS 16   // resident CTAs per SM its register budget is set for
+#define QESGD_DAA_MIN_CTAS 24   // resident CTAs per SM its register budget is set for
 #endif
 #ifndef QESGD_ENCODE_MIN_WARPS
 #define QESGD_ENCODE_MIN_WARPS 24  // resident warps per SM the register budget is set for
@@ -715,17 +715,6 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
     const uint32_t per_pass = 32u / nbw;                                 // workers per pass
     const float sf = (float)a.s;
 
-    float w[OPL][8];
-#pragma unroll
-    for (int o = 0; o < OPL; ++o) {
-        const uint64_t e0 = eb + 8u * o;
-        if (VEC && e0 + 8 <= a.d) {
-            ld256_rw(a.param + e0, w[o]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) w[o][j] = (e0 + j < a.d) ? a.param[e0 + j] : 0.0f;
-        }
-    }
     uint64_t acc[OPL][4];
 #pragma unroll
     for (int o = 0; o < OPL; ++o)
@@ -800,6 +789,19 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
         for (int i = 0; i < BATCH; ++i) {
             cw[i][0] = nx[i][0];
             cw[i][1] = nx[i][1];
+        }
+    }
+    // The parameter is fetched only now: its registers are not held through the worker loop
+    // (the other resident warps cover the latency), which lets more warps be resident.
+    float w[OPL][8];
+#pragma unroll
+    for (int o = 0; o < OPL; ++o) {
+        const uint64_t e0 = eb + 8u * o;
+        if (VEC && e0 + 8 <= a.d) {
+            ld256_rw(a.param + e0, w[o]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) w[o][j] = (e0 + j < a.d) ? a.param[e0 + j] : 0.0f;
         }
     }
     const float inv_k = a.avg_scale;   // alpha / K
