@@ -27,6 +27,8 @@ _lib.qesgd_ref_bucket_scale.argtypes = [_pf, _u32, _u32, _pd]
 _lib.qesgd_ref_bucket_scale.restype = _f32
 _lib.qesgd_ref_bucket_sumsq.argtypes = [_pf, _u32, _pd]
 _lib.qesgd_ref_bucket_sumsq.restype = C.c_double
+_lib.qesgd_ref_inv.argtypes = [_u32, _f32]
+_lib.qesgd_ref_inv.restype = _f32
 _lib.qesgd_ref_level.argtypes = [_f32, _f32, _u32, _u32]
 _lib.qesgd_ref_level.restype = _u32
 _lib.qesgd_ref_num_buckets.argtypes = [_u64, _u32]
@@ -95,6 +97,10 @@ def bucket_sumsq(z):
     z = np.ascontiguousarray(z, dtype=np.float32)
     scratch = np.zeros(z.size, dtype=np.float64)
     return float(_lib.qesgd_ref_bucket_sumsq(_f(z), z.size, scratch.ctypes.data_as(_pd)))
+
+
+def inv(s, scale):
+    return np.float32(_lib.qesgd_ref_inv(s, np.float32(scale)))
 
 
 def level(a, inv, s, h):

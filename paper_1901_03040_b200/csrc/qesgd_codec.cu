@@ -163,13 +163,21 @@ __device__ __forceinline__ uint64_t fma2_ru(uint64_t a, uint64_t b, uint64_t c) 
 // Two neighbouring elements at a time: the multiply and the fused multiply-add run on
 // packed pairs, the clamp stays scalar (it takes |.| for free).  x0, x1 receive the level
 // in bits 16..22 (what is below is of no interest).
+// CLIP: only a caller-given spacing can put |z|*inv above s.  With a scale taken from the
+// bucket itself |z| <= scale, and inv is s/scale rounded toward zero, so the exact product
+// is at most s and so is its fp32 rounding: the upper clamp would never act.
+template <bool CLIP>
 __device__ __forceinline__ void level_pair(float z0, float z1, uint64_t inv2, float sf,
                                            uint32_t h0, uint32_t h1, uint32_t &x0, uint32_t &x1)
 {
     float t0, t1;
     unpack2(mul2(pack2f(z0, z1), inv2), t0, t1);           // sign rides along, removed by |.|
-    const float r0 = fminf(fmaxf(fabsf(t0), 0x1p-30f), sf);
-    const float r1 = fminf(fmaxf(fabsf(t1), 0x1p-30f), sf);
+    float r0 = fmaxf(fabsf(t0), 0x1p-30f);
+    float r1 = fmaxf(fabsf(t1), 0x1p-30f);
+    if (CLIP) {
+        r0 = fminf(r0, sf);
+        r1 = fminf(r1, sf);
+    }
     float u0, u1;
     unpack2(fma2_ru(pack2f(r0, r1), pack2f(65536.0f, 65536.0f), pack2f(8388607.5f, 8388607.5f)),
             u0, u1);
@@ -407,7 +415,11 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
     {
         const bool nonfinite = !(my_scale <= 3.402823466e38f);   // Inf or NaN (scales are >= 0)
         const bool ok = !nonfinite && my_scale >= 0x1p-100f;
-        my_inv = ok ? __fdiv_rn(sf, my_scale) : 0.0f;
+        // s/scale rounded toward zero (keeps |z|*inv <= s): the nearest quotient, stepped
+        // down by one ulp when the exact residual s - q*scale says it lies above.
+        float q = __fdiv_rn(sf, my_scale);
+        if (__fmaf_rn(-q, my_scale, sf) < 0.0f) q = __uint_as_float(__float_as_uint(q) - 1u);
+        my_inv = ok ? q : 0.0f;
         my_scale = ok ? my_scale : 0.0f;
         if (REQ) my_delta = __fdiv_rn(my_scale, sf);   // grid spacing of the decoder
         // Lanes past the padded length hold zeros, so a set flag always belongs to real data.
@@ -454,7 +466,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
             Z[j + 1] = __float_as_uint(z[c][j + 1]);
             if (MODE == 2)   // NaN has no place on the grid: flagged (and encoded as 0 by the clamp)
                 flag |= (Z[j] & 0x7FFFFFFFu) > 0x7F800000u || (Z[j + 1] & 0x7FFFFFFFu) > 0x7F800000u;
-            level_pair(z[c][j], z[c][j + 1], inv2, sf, x[j >> 1] & 0xFFFFu, x[j >> 1] >> 16,
+            level_pair<MODE == 2>(z[c][j], z[c][j + 1], inv2, sf, x[j >> 1] & 0xFFFFu, x[j >> 1] >> 16,
                        X[j], X[j + 1]);
         }
         if (REQ) {

@@ -87,6 +87,26 @@ def test_rounding_probability_matches_eq4(v_over_delta):
         assert ups == 0                 # grid points never move
 
 
+def test_inverse_spacing_is_rounded_toward_zero_and_keeps_everything_in_range():
+    """inv is the largest float with inv * scale <= s (exact rationals); then fl32(|z| * inv) <= s
+    for every |z| <= scale, so the norm and max scales never reach Eq. 4's clipping branch."""
+    rng = np.random.default_rng(77)
+    for s in (1, 7, 100, 127):
+        for _ in range(200):
+            scale = np.float32(np.exp(rng.uniform(-40, 40)))
+            inv = q.inv(s, scale)
+            assert F(float(inv)) * F(float(scale)) <= s
+            assert F(float(np.nextafter(inv, np.float32(np.inf)))) * F(float(scale)) > s
+    for mode in (q.SCALE_NORM, q.SCALE_MAX):
+        for trial in range(20):
+            z = (rng.standard_normal(256) * np.exp(rng.uniform(-30, 30))).astype(np.float32)
+            if trial % 4 == 0:
+                z[1:] = 0                                  # a single element carries the whole norm
+            scale = q.bucket_scale(z, mode)
+            r = np.abs(z) * q.inv(127, scale)              # numpy fp32 multiply
+            assert r.dtype == np.float32 and r.max() <= np.float32(127)
+
+
 def test_level_monotone_in_draw_and_bounded():
     rng = np.random.default_rng(5)
     for s in (1, 7, 127):
@@ -289,15 +309,18 @@ def test_brute_force_expectation_small_d(mode, s, bits):
     zz[:d] = z
     _, scales, _ = q.encode(zz, None, 64, s, bits, mode, 0, 0, 0)
     scale = scales[0]
-    inv = np.float32(s) / scale
+    inv = q.inv(s, scale)
     floors, probs = [], []
     for i in range(d):
         lo, p, delta = _exact_up_probability(abs(z[i]), scale, s)
         lv = _levels_over_all_draws(abs(z[i]), inv, s)
-        freq = F(int((lv == lo + 1).sum()), 65536)
-        assert set(np.unique(lv)) <= {lo, lo + 1}
-        # 2^-17 from the draw resolution + one fp32 rounding of a*inv (<= r*2^-24)
-        assert abs(freq - p) <= F(1, 131072) + (lo + 1) * F(1, 1 << 23)
+        # the oracle rounds between the two grid points around its fp32 r = |z| * inv ...
+        r_fp = np.float32(abs(z[i])) * inv
+        assert set(np.unique(lv)) <= {math.floor(r_fp), math.floor(r_fp) + 1}
+        # ... and its mean level is the exact r = |z| / delta up to 2^-17 from the draw
+        # resolution and two fp32 roundings (inv and the product), each <= r * 2^-24
+        mean_level = F(int(lv.sum()), 65536)
+        assert abs(mean_level - (lo + p)) <= F(1, 131072) + (lo + 1) * F(1, 1 << 22)
         floors.append(lo)
         probs.append(p)
     mean = [F(0)] * d
