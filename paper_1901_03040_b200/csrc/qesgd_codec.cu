@@ -760,8 +760,16 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
             }
         }
     };
+    // One scale per lane and pass: lane L serves worker (first of the pass) + L / nbw, bucket
+    // bucket0 + L % nbw.  The scales of a pass are requested one pass ahead.
+    auto fetch_scale = [&](uint32_t kfirst) {
+        const uint32_t kk = kfirst + lane / nbw;
+        const uint64_t bb = bucket0 + (lane % nbw);
+        return (kk < a.K && bb < a.nb) ? __ldg(a.scales + (uint64_t)kk * a.scale_stride + bb) : 0.0f;
+    };
     uint32_t cw[BATCH][2], nx[BATCH][2];
     fetch(0u, cw);
+    float sc_next = fetch_scale(0u);
     float st = 0.0f;
     for (uint32_t kb = 0; kb < a.K; kb += BATCH) {
         fetch(kb + BATCH, nx);
@@ -770,11 +778,8 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
             const uint32_t k = kb + i;
             if (k < a.K) {   // uniform across the warp
                 if (k % per_pass == 0u) {   // a new pass: every lane computes one spacing
-                    const uint32_t kk = k + lane / nbw;
-                    const uint64_t bb = bucket0 + (lane % nbw);
-                    st = 0.0f;
-                    if (kk < a.K && bb < a.nb)
-                        st = __fdiv_rn(__ldg(a.scales + (uint64_t)kk * a.scale_stride + bb), sf);
+                    st = __fdiv_rn(sc_next, sf);
+                    sc_next = fetch_scale(k + per_pass);
                 }
                 const float step = __shfl_sync(FULL, st, (k % per_pass) * nbw + sub);
                 if (BITS == 4 && lut) {

@@ -222,9 +222,9 @@ def _assert_param_close(got, want, w_before, scales, bucket):
     assert (got != w_before).any()
 
 
-@pytest.mark.parametrize("K", [1, 2, 3, 8, 16, 33, 64])
-@pytest.mark.parametrize("bucket,bits,s", [(64, 4, 7), (128, 2, 1), (256, 2, 1), (512, 4, 7),
-                                           (2048, 8, 127), (8192, 4, 7)])
+@pytest.mark.parametrize("K", [1, 2, 3, 4, 5, 8, 16, 33, 64])
+@pytest.mark.parametrize("bucket,bits,s", [(64, 2, 1), (64, 4, 7), (64, 8, 127), (128, 2, 1), (256, 2, 1),
+                                           (512, 4, 7), (2048, 8, 127), (8192, 4, 7)])
 def test_decode_average_apply_matches_oracle(K, bucket, bits, s):
     n = 8192 * 2 + 300 + 5
     w, codes, scales = _daa_case(n, K, bucket, bits, s, seed=K * 7 + bits)
