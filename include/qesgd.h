@@ -22,7 +22,10 @@
  *     buffers must be 16-byte aligned and their per-worker strides multiples of
  *     16 bytes.
  *   - Calls enqueue work on the context's stream and return without waiting;
- *     only qesgd_status and qesgd_destroy synchronise.
+ *     only qesgd_status and qesgd_destroy synchronise.  The codec calls (encode,
+ *     encode_batch, requantize, decode, decode_average_apply/_axpy) do nothing but
+ *     launch kernels on that stream, so they may be recorded by CUDA stream capture
+ *     and replayed as a graph (worth it when a launch is as short as a host call).
  *   - Return value: QESGD_OK or a negative error code.  Nothing is enqueued
  *     when an error is returned.  No call aborts or throws.
  *   - Data problems (a non-finite value in a bucket) never fail a call: the

@@ -24,6 +24,13 @@ constexpr int CHUNK = 256;  // elements covered by one warp-wide 256-bit load
 #ifndef QESGD_DAA_BATCH
 #define QESGD_DAA_BATCH 4       // workers whose code words are fetched together
 #endif
+// chunks (64-bit code words per worker) a lane of that kernel owns, by code width
+#ifndef QESGD_DAA_WORDS_2BIT
+#define QESGD_DAA_WORDS_2BIT 1
+#endif
+#ifndef QESGD_DAA_WORDS_WIDE
+#define QESGD_DAA_WORDS_WIDE 2
+#endif
 #ifndef QESGD_DAA_MIN_CTAS
 #define QESGD_DAA_MIN_CTAS 24   // resident CTAs per SM its register budget is set for
 #endif
@@ -701,44 +708,51 @@ __device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], int o,
                       pack2(sg[2 * p], sg[2 * p + 1]), acc[p]);
 }
 
-// Every lane owns 8/BITS consecutive octets -- exactly one 64-bit code word per worker --
-// and a warp 256 * 8/BITS consecutive elements.  The grid spacings fl32(scale/s) a warp
+// A warp works on a tile of W chunks of 256 * 8/BITS consecutive elements.  In every
+// chunk a lane owns 8/BITS consecutive octets -- exactly one 64-bit code word per worker --
+// so a warp's loads of code words are contiguous.  The grid spacings fl32(scale/s) a warp
 // needs are computed once per warp (one division per lane) and handed out by shuffle;
 // code words are fetched several workers at a time so that independent loads are in
 // flight before the first is used.
-template <int BITS, bool VEC>
+template <int BITS, bool VEC, int W>
 __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
     qesgd_decode_average_apply_kernel(const DecodeArgs a)
 {
-    constexpr int OPL = 8 / BITS;                 // octets per lane: 4, 2, 1
+    constexpr int OPL = 8 / BITS;                 // octets per lane and chunk: 4, 2, 1
     constexpr int LANE_ELEMS = 8 * OPL;
-    constexpr uint32_t WCHUNK = 32 * LANE_ELEMS;  // elements per warp: 1024, 512, 256
-    constexpr uint32_t LOG2_WCHUNK = BITS == 2 ? 10 : (BITS == 4 ? 9 : 8);
-    constexpr int BATCH = QESGD_DAA_BATCH;
+    constexpr uint32_t WCHUNK = 32 * LANE_ELEMS;  // elements per chunk: 1024, 512, 256
+    constexpr uint32_t TILE = W * WCHUNK;         // elements per warp
+    constexpr uint32_t LOG2_TILE = (BITS == 2 ? 10 : (BITS == 4 ? 9 : 8)) + (W == 4 ? 2 : (W == 2 ? 1 : 0));
+    constexpr int BATCH = QESGD_DAA_BATCH / W > 0 ? QESGD_DAA_BATCH / W : 1;
     const uint32_t lane = threadIdx.x & 31u;
     const uint64_t warp_eb =
-        (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * (uint64_t)WCHUNK;
+        (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5) * (uint64_t)TILE;
     if (warp_eb >= a.d) return;  // whole warp out of range
-    const uint64_t eb = warp_eb + lane * (uint32_t)LANE_ELEMS;
     const uint32_t lb = a.log2_bucket;
-    const uint32_t nbw = lb >= LOG2_WCHUNK ? 1u : WCHUNK >> lb;          // buckets per warp: 1..16
-    const uint32_t sub = lb >= LOG2_WCHUNK ? 0u : (lane * (uint32_t)LANE_ELEMS) >> lb;
+    const uint32_t nbw = lb >= LOG2_TILE ? 1u : TILE >> lb;              // buckets per warp: 1..16
     const uint64_t bucket0 = warp_eb >> lb;
     const uint32_t per_pass = 32u / nbw;                                 // workers per pass
     const float sf = (float)a.s;
 
-    uint64_t acc[OPL][4];
+    uint64_t eb[W];      // first element of the lane in chunk c
+    uint32_t sub[W];     // its bucket, counted from the warp's first bucket
+    const uint8_t *__restrict__ cp[W];
+    uint64_t acc[W][OPL][4];
 #pragma unroll
-    for (int o = 0; o < OPL; ++o)
+    for (int c = 0; c < W; ++c) {
+        const uint32_t off = (uint32_t)c * WCHUNK + lane * (uint32_t)LANE_ELEMS;
+        eb[c] = warp_eb + off;
+        sub[c] = lb >= LOG2_TILE ? 0u : off >> lb;
+        // Lanes past the padded length of the streams read the warp's first word instead
+        // (their result is never stored), so no load needs a predicate.  The padded length
+        // is a multiple of 64, so a lane's 8, 16 or 32 elements are inside it or outside it.
+        const uint64_t safe_eb = eb[c] < (a.nb << lb) ? eb[c] : warp_eb;
+        cp[c] = reinterpret_cast<const uint8_t *>(a.codes) + (safe_eb >> 3) * (uint64_t)BITS;
 #pragma unroll
-        for (int p = 0; p < 4; ++p) acc[o][p] = 0ull;   // pairs of +0.0f
-
-    // Lanes past the padded length of the streams read the warp's first word instead
-    // (their result is never stored), so no load needs a predicate.  The padded length
-    // is a multiple of 64, so a lane's 8, 16 or 32 elements are inside it or outside it.
-    const uint64_t safe_eb = eb < (a.nb << lb) ? eb : warp_eb;
-    const uint8_t *__restrict__ cp =
-        reinterpret_cast<const uint8_t *>(a.codes) + (safe_eb >> 3) * (uint64_t)BITS;
+        for (int o = 0; o < OPL; ++o)
+#pragma unroll
+            for (int p = 0; p < 4; ++p) acc[c][o][p] = 0ull;   // pairs of +0.0f
+    }
 
     // Four-bit codes with buckets of at least 256 elements: a half-warp (16 lanes x 16
     // elements) lies inside one bucket, so the 16 possible code values +-level * step of a
@@ -748,15 +762,18 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
     const float signed_level = (lane & 8u) ? -(float)(lane & 7u) : (float)(lane & 7u);
 
     // Code words of BATCH workers are requested one batch ahead of the batch being decoded.
-    auto fetch = [&](uint32_t kfirst, uint32_t (&dst)[BATCH][2]) {
+    auto fetch = [&](uint32_t kfirst, uint32_t (&dst)[BATCH][W][2]) {
 #pragma unroll
         for (int i = 0; i < BATCH; ++i) {
-            dst[i][0] = dst[i][1] = 0u;
-            if (kfirst + i < a.K) {
-                const uint2 v = __ldg(reinterpret_cast<const uint2 *>(
-                    cp + (uint64_t)(kfirst + i) * a.code_stride));
-                dst[i][0] = v.x;
-                dst[i][1] = v.y;
+#pragma unroll
+            for (int c = 0; c < W; ++c) {
+                dst[i][c][0] = dst[i][c][1] = 0u;
+                if (kfirst + i < a.K) {
+                    const uint2 v = __ldg(reinterpret_cast<const uint2 *>(
+                        cp[c] + (uint64_t)(kfirst + i) * a.code_stride));
+                    dst[i][c][0] = v.x;
+                    dst[i][c][1] = v.y;
+                }
             }
         }
     };
@@ -767,7 +784,7 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
         const uint64_t bb = bucket0 + (lane % nbw);
         return (kk < a.K && bb < a.nb) ? __ldg(a.scales + (uint64_t)kk * a.scale_stride + bb) : 0.0f;
     };
-    uint32_t cw[BATCH][2], nx[BATCH][2];
+    uint32_t cw[BATCH][W][2], nx[BATCH][W][2];
     fetch(0u, cw);
     float sc_next = fetch_scale(0u);
     float st = 0.0f;
@@ -781,63 +798,73 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
                     st = __fdiv_rn(sc_next, sf);
                     sc_next = fetch_scale(k + per_pass);
                 }
-                const float step = __shfl_sync(FULL, st, (k % per_pass) * nbw + sub);
-                if (BITS == 4 && lut) {
-                    // every lane holds the value of code (lane & 15) for this worker; a code
-                    // is decoded by fetching its value from that lane of the same half-warp
-                    const float tab = __fmul_rn(signed_level, step);
 #pragma unroll
-                    for (int o = 0; o < OPL; ++o) {
-                        const uint32_t word = cw[i][o];
+                for (int c = 0; c < W; ++c) {
+                    const float step = __shfl_sync(FULL, st, (k % per_pass) * nbw + sub[c]);
+                    if (BITS == 4 && lut) {
+                        // every lane holds the value of code (lane & 15) for this worker; a
+                        // code is decoded by fetching its value from that lane of the same
+                        // half-warp
+                        const float tab = __fmul_rn(signed_level, step);
 #pragma unroll
-                        for (int p = 0; p < 4; ++p) {
-                            const float v0 = __shfl_sync(FULL, tab, (int)(word >> (8 * p)), 16);
-                            const float v1 = __shfl_sync(FULL, tab, (int)(word >> (8 * p + 4)), 16);
-                            acc[o][p] = add2(acc[o][p], pack2f(v0, v1));
+                        for (int o = 0; o < OPL; ++o) {
+                            const uint32_t word = cw[i][c][o];
+#pragma unroll
+                            for (int p = 0; p < 4; ++p) {
+                                const float v0 = __shfl_sync(FULL, tab, (int)(word >> (8 * p)), 16);
+                                const float v1 = __shfl_sync(FULL, tab, (int)(word >> (8 * p + 4)), 16);
+                                acc[c][o][p] = add2(acc[c][o][p], pack2f(v0, v1));
+                            }
                         }
-                    }
-                } else {
+                    } else {
 #pragma unroll
-                    for (int o = 0; o < OPL; ++o) accumulate_octet<BITS>(cw[i], o, step, acc[o]);
+                        for (int o = 0; o < OPL; ++o)
+                            accumulate_octet<BITS>(cw[i][c], o, step, acc[c][o]);
+                    }
                 }
             }
         }
 #pragma unroll
-        for (int i = 0; i < BATCH; ++i) {
-            cw[i][0] = nx[i][0];
-            cw[i][1] = nx[i][1];
-        }
+        for (int i = 0; i < BATCH; ++i)
+#pragma unroll
+            for (int c = 0; c < W; ++c) {
+                cw[i][c][0] = nx[i][c][0];
+                cw[i][c][1] = nx[i][c][1];
+            }
     }
     // The parameter is fetched only now: its registers are not held through the worker loop
     // (the other resident warps cover the latency), which lets more warps be resident.
-    float w[OPL][8];
-#pragma unroll
-    for (int o = 0; o < OPL; ++o) {
-        const uint64_t e0 = eb + 8u * o;
-        if (VEC && e0 + 8 <= a.d) {
-            ld256_rw(a.param + e0, w[o]);
-        } else {
-#pragma unroll
-            for (int j = 0; j < 8; ++j) w[o][j] = (e0 + j < a.d) ? a.param[e0 + j] : 0.0f;
-        }
-    }
     const float inv_k = a.avg_scale;   // alpha / K
 #pragma unroll
-    for (int o = 0; o < OPL; ++o) {
+    for (int c = 0; c < W; ++c) {
+        float w[OPL][8];
 #pragma unroll
-        for (int p = 0; p < 4; ++p) {
-            float lo, hi;
-            unpack2(acc[o][p], lo, hi);
-            w[o][2 * p] = __fmaf_rn(lo, inv_k, w[o][2 * p]);
-            w[o][2 * p + 1] = __fmaf_rn(hi, inv_k, w[o][2 * p + 1]);
+        for (int o = 0; o < OPL; ++o) {
+            const uint64_t e0 = eb[c] + 8u * o;
+            if (VEC && e0 + 8 <= a.d) {
+                ld256_rw(a.param + e0, w[o]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) w[o][j] = (e0 + j < a.d) ? a.param[e0 + j] : 0.0f;
+            }
         }
-        const uint64_t e0 = eb + 8u * o;
-        if (VEC && e0 + 8 <= a.d) {
-            st256(a.param + e0, w[o]);
-        } else {
 #pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (e0 + j < a.d) a.param[e0 + j] = w[o][j];
+        for (int o = 0; o < OPL; ++o) {
+#pragma unroll
+            for (int p = 0; p < 4; ++p) {
+                float lo, hi;
+                unpack2(acc[c][o][p], lo, hi);
+                w[o][2 * p] = __fmaf_rn(lo, inv_k, w[o][2 * p]);
+                w[o][2 * p + 1] = __fmaf_rn(hi, inv_k, w[o][2 * p + 1]);
+            }
+            const uint64_t e0 = eb[c] + 8u * o;
+            if (VEC && e0 + 8 <= a.d) {
+                st256(a.param + e0, w[o]);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j)
+                    if (e0 + j < a.d) a.param[e0 + j] = w[o][j];
+            }
         }
     }
 }
@@ -925,13 +952,14 @@ int QESGD_CAT(qesgd_launch_decode_, QESGD_BITS)(const DecodeArgs &a, bool vec, c
 int QESGD_CAT(qesgd_launch_decode_average_apply_, QESGD_BITS)(const DecodeArgs &a, bool vec,
                                                               cudaStream_t stream)
 {
-    const uint64_t warp_elems = 256ull * (8u / QESGD_BITS);   // one warp each (see the kernel)
+    constexpr int W = QESGD_BITS == 2 ? QESGD_DAA_WORDS_2BIT : QESGD_DAA_WORDS_WIDE;
+    const uint64_t warp_elems = 256ull * (8u / QESGD_BITS) * W;   // one tile per warp (see the kernel)
     const uint64_t warps = (a.d + warp_elems - 1) / warp_elems;
     const uint64_t wpc = QESGD_DAA_THREADS / 32;
     const uint64_t blocks = (warps + wpc - 1) / wpc;
     if (blocks == 0 || blocks > 0x7FFFFFFFull) return (int)cudaErrorInvalidValue;
     dim3 grid((unsigned)blocks), block(QESGD_DAA_THREADS);
-    if (vec) qesgd_decode_average_apply_kernel<QESGD_BITS, true><<<grid, block, 0, stream>>>(a);
-    else qesgd_decode_average_apply_kernel<QESGD_BITS, false><<<grid, block, 0, stream>>>(a);
+    if (vec) qesgd_decode_average_apply_kernel<QESGD_BITS, true, W><<<grid, block, 0, stream>>>(a);
+    else qesgd_decode_average_apply_kernel<QESGD_BITS, false, W><<<grid, block, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }

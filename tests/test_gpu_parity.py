@@ -429,3 +429,45 @@ def test_invalid_arguments_return_einval_and_launch_nothing():
     c.qesgd_decode_average_apply(z, 0, 3, codes, 0, scales, 0, 512, 7, 4)
     assert c.qesgd_launch_count() == before
     assert c.qesgd_status() == 0
+
+
+# ----------------------------------------------------------- graph replay ----
+def test_round_recorded_into_a_cuda_graph_replays_bit_identically():
+    """The codec calls only enqueue kernels on the context's stream, so a round (encode of all
+    workers, then decode-average-apply) can be recorded by stream capture; replaying the graph
+    must give exactly what the direct calls give."""
+    K, d, bucket, s, bits = 4, 3 * 4096 + 77, 256, 7, 4
+    stream = torch.cuda.Stream()
+    ctx = qesgd.Context(0, stream)
+    stride = (d + 7) // 8 * 8
+    anchor = G.dev(synthetic.anchor_vector(d, seed=5))
+    locs = torch.zeros((K, stride), dtype=torch.float32, device="cuda")
+    for k in range(K):
+        locs[k, :d] = anchor + G.dev(_delta(d, seed=60 + k))
+    codes, scales = qesgd.alloc_stream_buffers(K, d, bucket, bits, "cuda")
+
+    def one_round(param):
+        ctx.qesgd_encode_batch(locs, stride, anchor, d, K, bucket, s, bits, qesgd.SCALE_NORM, 11, 0, 2,
+                               codes, codes.stride(0), scales, scales.stride(0))
+        ctx.qesgd_decode_average_apply(param, d, K, codes, codes.stride(0), scales, scales.stride(0),
+                                       bucket, s, bits)
+    direct = anchor.clone()
+    torch.cuda.synchronize()
+    one_round(direct)
+    stream.synchronize()
+    want_codes, want_scales = codes.clone(), scales.clone()
+    codes.zero_()
+    scales.zero_()
+    replayed = anchor.clone()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=stream):
+        one_round(replayed)
+    assert (codes == 0).all()                     # capture records, it does not run
+    with torch.cuda.stream(stream):
+        graph.replay()
+    stream.synchronize()
+    assert ctx.qesgd_status() == 0
+    assert torch.equal(codes, want_codes) and torch.equal(scales, want_scales)
+    assert torch.equal(replayed, direct)
+    ctx.close()
