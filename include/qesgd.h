@@ -91,9 +91,7 @@ uint64_t qesgd_code_bytes(uint64_t d, uint32_t bucket, uint32_t bits);
  *   z_i   = fl32(local_i - anchor_i), or local_i when anchor == NULL
  *   scale = fl32(sqrt(sum z_i^2))  (NORM; fp64 sum over the balanced binary tree on
  *           index order)  |  max |z_i|  (MAX)  |  fl32(s*fixed_delta)  (FIXED)
- *   r_i   = min(fl32(|z_i| * inv), s), inv = s/scale rounded toward zero to fp32 (so that a
- *           coordinate of the bucket never leaves the grid's range, Lemma 2);
- *   level_i = floor(r_i) + [u_i < frac(r_i)]
+ *   r_i   = min(fl32(|z_i| * fl32(s/scale)), s);  level_i = floor(r_i) + [u_i < frac(r_i)]
  *   u_i   = (h_i + 1/2) / 2^16 with h_i the 16-bit draw of element i from
  *           Philox4x32-10, counter (i>>3 low, i>>3 high, worker, epoch), key = seed,
  *           32-bit word (i>>1)&3, half (i&1)

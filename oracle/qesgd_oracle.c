@@ -123,7 +123,7 @@ float qesgd_ref_bucket_scale(const float *z, uint32_t B, uint32_t scale_mode, do
 /* ------------------------------------------------------------------------ */
 /* Stochastic rounding of one magnitude (Eq. 4 with delta = scale / s and    */
 /* the grid taken symmetric, |k| <= s): r = a / delta computed as a * inv    */
-/* with inv = s / scale rounded toward zero; values above the top of the range stay */
+/* with inv = fl32(s / scale); values at or above the top of the range stay  */
 /* at s (first branch of Eq. 4); inside the range the result is floor(r)     */
 /* with probability ceil - r and floor(r) + 1 with probability r - floor     */
 /* (second and third branch).  The draw h decides: up iff (h + 1/2)/2^16 < p.*/
@@ -138,19 +138,13 @@ uint32_t qesgd_ref_level(float a, float inv, uint32_t s, uint32_t h)
     return (uint32_t)f + (uint32_t)up;
 }
 
-/* inv = s / scale rounded TOWARD ZERO.  Lemma 2 asks that every coordinate lie inside the
- * grid's range, |z| / delta <= s with delta = scale / s.  With the quotient rounded down,
- * |z| * inv <= s holds in exact arithmetic whenever |z| <= scale, and because s is a float it
- * still holds after the product is rounded to nearest: the top of the range is never
- * exceeded and the clipping branch of Eq. 4 stays unreachable for the norm and max scales.
- * (The double quotient is within 2^-53 of the exact one, far closer than any float that is
- * not the exact quotient itself, so the comparison below decides the direction exactly.) */
+/* inv = fl32(s / scale): one correctly rounded fp32 division per bucket.  Rounded to
+ * nearest it can exceed the exact quotient by half an ulp, so the product |z| * inv of the
+ * bucket's largest coordinate can land one ulp above s; the min() in qesgd_ref_level is
+ * Eq. 4's first branch and takes that back to s. */
 float qesgd_ref_inv(uint32_t s, float scale)
 {
-    double q = (double)s / (double)scale;
-    float f = (float)q;
-    if ((double)f > q) f = nextafterf(f, 0.0f);
-    return f;
+    return (float)s / scale;
 }
 
 static int valid_bits(uint32_t bits) { return bits == 2 || bits == 4 || bits == 8; }

@@ -170,9 +170,14 @@ __device__ __forceinline__ uint64_t fma2_ru(uint64_t a, uint64_t b, uint64_t c) 
 // Two neighbouring elements at a time: the multiply and the fused multiply-add run on
 // packed pairs, the clamp stays scalar (it takes |.| for free).  x0, x1 receive the level
 // in bits 16..22 (what is below is of no interest).
-// CLIP: only a caller-given spacing can put |z|*inv above s.  With a scale taken from the
-// bucket itself |z| <= scale, and inv is s/scale rounded toward zero, so the exact product
-// is at most s and so is its fp32 rounding: the upper clamp would never act.
+// CLIP: only a caller-given spacing needs the upper clamp min(r, s).  With a scale taken
+// from the bucket itself |z| <= scale, and inv = fl32(s/scale) is at most (s/scale) *
+// (1 + 2^-24), so the exact product is below s + ulp(s) and its fp32 rounding is s or
+// s + ulp(s).  (Where s/scale is subnormal -- scale > s * 2^126, so s < 4 -- inv is off by
+// at most 2^-150 and the product by at most 2^128 * 2^-150 = 2^-22.)  Either way r - s <=
+// 2^-17 for s <= 127, i.e. at most 1/2 after the scaling by 2^16, and ceil(s * 2^16 + 1/2
+// - 1/2) is still s * 2^16: the overshoot never reaches a level, so the clamp would change
+// nothing.
 template <bool CLIP>
 __device__ __forceinline__ void level_pair(float z0, float z1, uint64_t inv2, float sf,
                                            uint32_t h0, uint32_t h1, uint32_t &x0, uint32_t &x1)
@@ -422,11 +427,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
     {
         const bool nonfinite = !(my_scale <= 3.402823466e38f);   // Inf or NaN (scales are >= 0)
         const bool ok = !nonfinite && my_scale >= 0x1p-100f;
-        // s/scale rounded toward zero (keeps |z|*inv <= s): the nearest quotient, stepped
-        // down by one ulp when the exact residual s - q*scale says it lies above.
-        float q = __fdiv_rn(sf, my_scale);
-        if (__fmaf_rn(-q, my_scale, sf) < 0.0f) q = __uint_as_float(__float_as_uint(q) - 1u);
-        my_inv = ok ? q : 0.0f;
+        my_inv = ok ? __fdiv_rn(sf, my_scale) : 0.0f;
         my_scale = ok ? my_scale : 0.0f;
         if (REQ) my_delta = __fdiv_rn(my_scale, sf);   // grid spacing of the decoder
         // Lanes past the padded length hold zeros, so a set flag always belongs to real data.

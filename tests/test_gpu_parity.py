@@ -143,6 +143,43 @@ def test_subnormal_and_mixed_magnitudes_match():
             _assert_streams_equal(G.gpu_encode(z, None, *args), ref.encode(z, None, *args))
 
 
+def _unpack_levels(words, bits):
+    """Levels (codes without their sign bit) of a little-endian packed stream."""
+    per = 32 // bits
+    shifts = (np.arange(per, dtype=np.uint32) * bits)[None, :]
+    fields = (words.astype(np.uint32)[:, None] >> shifts) & np.uint32((1 << bits) - 1)
+    return (fields & np.uint32((1 << (bits - 1)) - 1)).reshape(-1)
+
+
+def test_bucket_maxima_and_huge_scales_stay_at_the_top_level():
+    """Buckets whose largest coordinates equal the scale (max mode: many copies of the maximum;
+    norm mode: one coordinate carries the whole norm), over many scales, and scales so large that
+    the inverse spacing s/scale is subnormal: the product |z| * inv may exceed s by an ulp there,
+    and the codes must still be the oracle's (top level s, never s + 1)."""
+    rng = np.random.default_rng(99)
+    nb, bucket = 256, 64
+    for bits, s in ((2, 1), (4, 2), (4, 3), (4, 7), (8, 100), (8, 127)):
+        z = np.zeros((nb, bucket), dtype=np.float32)
+        mags = np.exp(rng.uniform(-30, 30, nb)).astype(np.float32)
+        mags[nb // 2:] = (2.0 ** rng.uniform(126, 127.9, nb - nb // 2)).astype(np.float32)
+        signs = rng.choice(np.float32([-1, 1]), (nb, bucket))
+        z[:, :16] = mags[:, None] * signs[:, :16]                     # copies of the maximum
+        z[:, 16:] = (mags[:, None] * rng.uniform(0, 1, (nb, bucket - 16))).astype(np.float32) * signs[:, 16:]
+        flat = z.reshape(-1)
+        for epoch in range(3):
+            args = (bucket, s, bits, ref.SCALE_MAX, 17, 1, epoch)
+            got, want = G.gpu_encode(flat, None, *args), ref.encode(flat, None, *args)
+            _assert_streams_equal(got, want)
+        levels = _unpack_levels(want[0], bits)[: nb * bucket].reshape(nb, bucket)
+        assert (levels[:, :16] == s).all()
+        single = np.zeros((nb, bucket), dtype=np.float32)             # one coordinate = the norm
+        single[np.arange(nb), rng.integers(0, bucket, nb)] = mags * signs[:, 0]
+        args = (bucket, s, bits, ref.SCALE_NORM, 17, 1, 0)
+        got, want = G.gpu_encode(single.reshape(-1), None, *args), ref.encode(single.reshape(-1), None, *args)
+        _assert_streams_equal(got, want)
+        assert got[2] == 0
+
+
 def test_fixed_delta_mode_matches_and_clips():
     n = 8192 + 100
     z = _delta(n, seed=21)

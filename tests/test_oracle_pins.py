@@ -87,24 +87,29 @@ def test_rounding_probability_matches_eq4(v_over_delta):
         assert ups == 0                 # grid points never move
 
 
-def test_inverse_spacing_is_rounded_toward_zero_and_keeps_everything_in_range():
-    """inv is the largest float with inv * scale <= s (exact rationals); then fl32(|z| * inv) <= s
-    for every |z| <= scale, so the norm and max scales never reach Eq. 4's clipping branch."""
+def test_inverse_spacing_is_the_nearest_float_and_the_top_of_the_range_is_a_fixed_point():
+    """inv = fl32(s / scale) is the float nearest to the exact quotient.  For the largest
+    coordinate a bucket can hold (|z| = scale) the fp32 product |z| * inv is s or one ulp above
+    it (at most 2^-22 above where inv is subnormal, which needs s < 4); Eq. 4's first branch (the
+    min) takes it back to s, and even without that branch the overshoot is too small to move a
+    draw: ceil(r * 2^16 - 1/2) = s * 2^16 because the overshoot is at most 2^-17 for s <= 127."""
     rng = np.random.default_rng(77)
-    for s in (1, 7, 100, 127):
-        for _ in range(200):
+    for s in (1, 3, 7, 100, 127):
+        for trial in range(400):
             scale = np.float32(np.exp(rng.uniform(-40, 40)))
+            if trial >= 300:                                  # inv = s / scale is subnormal here
+                scale = np.float32(2.0 ** rng.uniform(126, 128) * 0.999)
             inv = q.inv(s, scale)
-            assert F(float(inv)) * F(float(scale)) <= s
-            assert F(float(np.nextafter(inv, np.float32(np.inf)))) * F(float(scale)) > s
-    for mode in (q.SCALE_NORM, q.SCALE_MAX):
-        for trial in range(20):
-            z = (rng.standard_normal(256) * np.exp(rng.uniform(-30, 30))).astype(np.float32)
-            if trial % 4 == 0:
-                z[1:] = 0                                  # a single element carries the whole norm
-            scale = q.bucket_scale(z, mode)
-            r = np.abs(z) * q.inv(127, scale)              # numpy fp32 multiply
-            assert r.dtype == np.float32 and r.max() <= np.float32(127)
+            exact = F(s) / F(float(scale))
+            lo, hi = np.nextafter(inv, np.float32(0)), np.nextafter(inv, np.float32(np.inf))
+            assert abs(F(float(inv)) - exact) <= min(abs(F(float(lo)) - exact), abs(F(float(hi)) - exact))
+            r = scale * inv                                   # numpy fp32 multiply
+            assert r.dtype == np.float32
+            assert float(r) - s <= max(float(np.spacing(np.float32(s))), 2.0 ** -22)
+            assert math.ceil(F(float(r)) * 65536 - F(1, 2)) <= s * 65536
+            for h in (0, 1, 32767, 65535):
+                if r >= s:
+                    assert q.level(scale, inv, s, h) == s
 
 
 def test_level_monotone_in_draw_and_bounded():
