@@ -593,8 +593,11 @@ def run_c1(args, device, world, rank):
             "gpu_launches": int(ctx.qesgd_launch_count() - launches0),
             "kernels": {k: {"avg_ms": statistics.mean(v)} for k, v in times.items()},
             "x_bytes_per_epoch": int(n * d * 4),
-            "local_epoch_gbs": 2.0 * n * d * 4 / (statistics.mean(times["local_epoch"]) * 1e-3) / 1e9,
-            "loss_before": loss0, "loss_after_rounds": losses}
+            # algorithmic bytes of the epoch: every row of X once (the minibatch stays on chip
+            # between the margin pass and the update pass)
+            "local_epoch_gbs": n * d * 4 / (statistics.mean(times["local_epoch"]) * 1e-3) / 1e9,
+            "loss_before": loss0, "loss_after_first_rounds": losses[:3], "loss_after_last_round": losses[-1],
+            "rounds": len(losses)}
     if rank == 0:
         print(json.dumps(line))
 

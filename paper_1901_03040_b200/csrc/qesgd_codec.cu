@@ -197,17 +197,45 @@ __device__ __forceinline__ void level_pair(float z0, float z1, uint64_t inv2, fl
     x1 = __float_as_uint(u1) - h1 + (65535u - 0x4B000000u);
 }
 
+// (a & b) | c and (a & b) ^ c as one three-input logic operation each
+__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+__device__ __forceinline__ uint32_t and_xor(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
 // Packing.  X[j] holds the level of element j in byte 2 (bits 16..22) and Z[j] the
 // sign of z_j in bit 31.  Bytes are gathered with PRMT, fields merged with
 // multiply-adds; the sign is kept only where the level is not zero, which is
 // tested on whole words (a field plus its largest level never carries).
+// X[j] = U + 65535 - h lies in [0, 2^23), so its byte 3 is always zero and serves as the
+// source of zero bytes.  PRMT's replicate mode (selector nibble 8 + n) turns the top bit of
+// byte n into a whole byte of ones or zeros, so a sign lands on any bit of its byte by a
+// mask alone, without a shift.
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
 __device__ __forceinline__ uint32_t bytes2(uint32_t a, uint32_t b)   // [a.b2, b.b2, 0, 0]
 {
-    return __byte_perm(a, b, 0x0062) & 0xFFFFu;
+    return prmt(a, b, 0x3362u);
 }
 __device__ __forceinline__ uint32_t bytes3(uint32_t a, uint32_t b)   // [a.b3, b.b3, ., .]
 {
     return __byte_perm(a, b, 0x0073);
+}
+__device__ __forceinline__ uint32_t signs2(uint32_t a, uint32_t b)   // [a<0 ? FF : 00, b<0 ? FF : 00, ., .]
+{
+    return prmt(a, b, 0x00FBu);
 }
 
 template <int BITS>
@@ -228,9 +256,9 @@ __device__ __forceinline__ void pack_octet(const uint32_t (&X)[8], const uint32_
         const uint32_t le = __byte_perm(__byte_perm(X[0], X[2], 0x0062), __byte_perm(X[4], X[6], 0x0062), 0x5410);
         const uint32_t lo = __byte_perm(__byte_perm(X[1], X[3], 0x0062), __byte_perm(X[5], X[7], 0x0062), 0x5410);
         const uint32_t lv = le + lo * 16u;
-        const uint32_t se = __byte_perm(bytes3(Z[0], Z[2]), bytes3(Z[4], Z[6]), 0x5410);
-        const uint32_t so = __byte_perm(bytes3(Z[1], Z[3]), bytes3(Z[5], Z[7]), 0x5410);
-        const uint32_t sg = ((se >> 4) & 0x08080808u) | (so & 0x80808080u);
+        const uint32_t se = __byte_perm(signs2(Z[0], Z[2]), signs2(Z[4], Z[6]), 0x5410);
+        const uint32_t so = __byte_perm(signs2(Z[1], Z[3]), signs2(Z[5], Z[7]), 0x5410);
+        const uint32_t sg = and_or(se, 0x08080808u, so & 0x80808080u);
         out[0] = lv | (sg & (lv + 0x77777777u));
         out[1] = 0u;
     } else {
@@ -238,10 +266,9 @@ __device__ __forceinline__ void pack_octet(const uint32_t (&X)[8], const uint32_
         const uint32_t g0 = bytes2(X[0], X[4]), g1 = bytes2(X[1], X[5]);
         const uint32_t g2 = bytes2(X[2], X[6]), g3 = bytes2(X[3], X[7]);
         const uint32_t lv = (g0 + g1 * 4u) + (g2 * 16u + g3 * 64u);
-        const uint32_t h0 = bytes3(Z[0], Z[4]), h1 = bytes3(Z[1], Z[5]);
-        const uint32_t h2 = bytes3(Z[2], Z[6]), h3 = bytes3(Z[3], Z[7]);
-        const uint32_t sg = ((h0 >> 6) & 0x0202u) | ((h1 >> 4) & 0x0808u) | ((h2 >> 2) & 0x2020u) |
-                            (h3 & 0x8080u);
+        const uint32_t h0 = signs2(Z[0], Z[4]), h1 = signs2(Z[1], Z[5]);
+        const uint32_t h2 = signs2(Z[2], Z[6]), h3 = signs2(Z[3], Z[7]);
+        const uint32_t sg = and_or(h3, 0x8080u, and_or(h2, 0x2020u, and_or(h1, 0x0808u, h0 & 0x0202u)));
         out[0] = lv | (sg & (lv << 1));
         out[1] = 0u;
     }
@@ -639,19 +666,6 @@ __global__ void __launch_bounds__(256) qesgd_decode_kernel(const DecodeArgs a)
 }
 
 // -------------------------------------------- decode + average + apply ------
-// (a & b) | c and (a & b) ^ c as one three-input logic operation each
-__device__ __forceinline__ uint32_t and_or(uint32_t a, uint32_t b, uint32_t c)
-{
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
-__device__ __forceinline__ uint32_t and_xor(uint32_t a, uint32_t b, uint32_t c)
-{
-    uint32_t d;
-    asm("lop3.b32 %0, %1, %2, %3, 0x6A;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
-    return d;
-}
 
 // acc += +-level * step for the 8 codes of one octet, two elements per arithmetic
 // instruction (acc[p] holds elements 2p, 2p+1).  One rounding per product-sum: the sign
