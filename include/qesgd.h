@@ -61,6 +61,7 @@ extern "C" {
 #define QESGD_SCALE_FIXED 2u /* scale = s*delta with the grid spacing delta given  */
 
 #define QESGD_STATUS_NONFINITE 1u /* a bucket held NaN/Inf or its norm overflowed fp32 */
+#define QESGD_STATUS_TIMEOUT 2u   /* a bounded wait inside the local-epoch kernel ran out   */
 
 #define QESGD_MAX_WORKERS 64u
 #define QESGD_MIN_BUCKET 64u
@@ -187,8 +188,18 @@ int qesgd_lr_gradient(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32_t
 int qesgd_lr_local_epoch(qesgd_ctx *ctx, const float *X, const float *y, uint64_t n_local,
                          uint64_t d, uint32_t batch, float lr, float *u);
 /* K workers side by side: worker k owns rows [k*n_local, (k+1)*n_local) of X and
- * y and updates u + k*u_stride (elements).  Step t of every worker runs in the
- * same launches. */
+ * y and updates u + k*u_stride (elements).
+ * Where the shape allows (d a multiple of 4 and at most 512 columns per SM, minibatches
+ * of at most 256 rows, X and u 16-byte aligned, u_stride a multiple of 4) the whole epoch
+ * of all K workers is ONE persistent kernel, launched cooperatively with one CTA per SM,
+ * that stages every minibatch in shared memory by TMA and reads X from HBM once; its
+ * CTAs exchange partial margins through the context's workspace, which the call clears
+ * first.  Every wait inside it is bounded (about a second): should one run out, the
+ * kernel returns, u is left partly updated and QESGD_STATUS_TIMEOUT is set in the status
+ * word.  The kernel needs all its CTAs resident at once, so do not run it next to other
+ * kernels that occupy the device for long.  Other shapes run one margin pass and one
+ * update pass per minibatch, step t of every worker in the same launches.  Results are
+ * deterministic (fixed summation order) on either path. */
 int qesgd_lr_local_epoch_batch(qesgd_ctx *ctx, const float *X, const float *y, uint64_t n_local,
                                uint64_t d, uint32_t K, uint32_t batch, float lr, float *u,
                                uint64_t u_stride);

@@ -22,6 +22,7 @@ UNITS = [
     ("qesgd_codec.cu", "qesgd_codec_4.o", ["-fmad=false", "-DQESGD_BITS=4"]),
     ("qesgd_codec.cu", "qesgd_codec_8.o", ["-fmad=false", "-DQESGD_BITS=8"]),
     ("qesgd_lr.cu", "qesgd_lr.o", []),
+    ("qesgd_lr_epoch.cu", "qesgd_lr_epoch.o", []),
     ("qesgd_api.cu", "qesgd_api.o", []),
 ]
 

@@ -292,6 +292,15 @@ int qesgd_lr_local_epoch_batch(qesgd_ctx *ctx, const float *X, const float *y, u
     if ((uint64_t)K * m_max > ctx->lr_work_floats) return QESGD_EINVAL;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
+    {   // the whole epoch in one persistent kernel where its shape allows
+        int launched = 0;
+        const int e = qesgd_launch_lr_epoch_fused(X, y, n_local, d, K, batch, lr, u, K > 1 ? u_stride : 0,
+                                                  ctx->d_lr_work, ctx->lr_work_floats, ctx->d_status,
+                                                  ctx->device, ctx->sm_count, ctx->stream, &launched);
+        ctx->launches += (uint64_t)launched;
+        if (e > 0) return cuda_fail(ctx, e);
+        if (e == 0) return QESGD_OK;
+    }
     for (uint64_t r = 0; r < n_local; r += batch) {
         const uint32_t m = (uint32_t)(n_local - r < batch ? n_local - r : batch);
         int launched = 0;

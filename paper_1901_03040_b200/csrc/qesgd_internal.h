@@ -103,3 +103,11 @@ int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float 
 int qesgd_launch_lr_gradient(const float *Xb, const float *yb, uint32_t m, uint64_t d,
                              const float *w, float *g, float *work, uint64_t work_floats,
                              cudaStream_t stream, int *launched);
+// A whole local epoch of K workers as one persistent kernel that keeps each minibatch in
+// shared memory between its two uses.  Returns 0 = launched (one memset + one kernel),
+// -1 = shape not covered (the caller falls back to qesgd_launch_lr_step per minibatch),
+// > 0 = cudaError_t.  `work` is zeroed and used for the inter-CTA counters and partial margins.
+int qesgd_launch_lr_epoch_fused(const float *X, const float *y, uint64_t n_local, uint64_t d,
+                                uint32_t K, uint32_t batch, float lr, float *u, uint64_t u_stride,
+                                float *work, uint64_t work_floats, uint32_t *status, int device,
+                                int sm_count, cudaStream_t stream, int *launched);

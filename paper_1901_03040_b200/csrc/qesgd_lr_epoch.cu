@@ -1,0 +1,591 @@
+// Local epoch of logistic-regression minibatch SGD as ONE persistent kernel for sm_100a
+// (paper Sec. 1: f_i(w) = log(1 + exp(-y_i x_i^T w)); Eq. 2: u <- u - (lr/m) sum_j grad f_j(u);
+// worker task of Algorithm 3: consecutive minibatches of the worker's shard).
+//
+// A step needs the minibatch twice -- once for the margins x_j . u, once for the update
+// sum_j c_j x_j -- with a reduction over all columns in between.  Here every CTA owns a
+// slice of `cols` columns for the whole epoch and keeps its slice of each minibatch in
+// shared memory between the two uses, so X is read from HBM exactly once:
+//
+//   tile (t, k)  = minibatch t of worker k; tiles are processed t-major, k-minor, and
+//                  alternate between two shared-memory buffers
+//   sub-tile     = SUB rows of a tile's column slice, fetched by TMA (one or two 2-D boxes,
+//                  cp.async.bulk.tensor global -> shared, completion on an mbarrier per
+//                  sub-tile); a producer warp issues the copies of tile i+2 as soon as the
+//                  consumer warps have released the buffer of tile i
+//   M(i)  margins of tile i over the CTA's columns -> partial[i % RING][row][cta],
+//         then fence + one atomic increment of counter[i]
+//   W(i)  wait until counter[i] == number of CTAs, sum the partials of every row in a
+//         fixed order, coefficients (lr/m) y_j / (1 + exp(y_j m_j)) into shared memory
+//   U(i)  u[cols] += sum_j coef_j x_j from the buffer, then the buffer is released
+//
+// Each tile's M, W, U is a chain of dependent round trips to global memory (fence, count,
+// partial margins) that lasts longer than the tile's own transfer from HBM.  The eight
+// consumer warps therefore form two groups of four; group g owns buffer g and the tiles
+// g, g+2, g+4, ... and runs M(i), W(i), U(i) for them, so one group computes while the other
+// waits, and the copies of the tile after next are in flight meanwhile.  A worker's
+// consecutive minibatches are K tiles apart: with an even K they stay in one group, with an
+// odd K a group waits for the other group's update before it takes the margins.
+//
+// The CTAs wait on one another, so the kernel is launched cooperatively (all CTAs are
+// resident by construction: at most one per SM).  Every wait is bounded: a wait that
+// runs out sets QESGD_STATUS_TIMEOUT and an abort word that the other CTAs poll; each CTA
+// then waits (bounded again) for its own copies in flight and returns.
+#include <cuda.h>
+
+#include <mutex>
+
+#include "qesgd_internal.h"
+
+namespace {
+
+constexpr int EP_CONSUMERS = 256;                 // 8 consumer warps
+constexpr int EP_GROUP = EP_CONSUMERS / 2;        // two groups of 4 warps, one per tile buffer
+constexpr int EP_THREADS = EP_CONSUMERS + 32;     // + 1 producer warp
+constexpr int SUB = 8;               // rows per sub-tile
+constexpr int EP_RING = 8;           // partial-margin slots; CTAs are at most 2 tiles apart
+constexpr int EP_MAX_COLS = 512;     // columns per CTA: 128 groups of 4
+constexpr int EP_BOX_COLS = 256;     // widest TMA box
+constexpr int EP_MAX_M = 256;        // rows per minibatch the fused path takes
+constexpr int EP_MAX_NSUB = EP_MAX_M / SUB;
+#ifndef EP_INFLIGHT
+#define EP_INFLIGHT 3               // sub-tiles a CTA has outstanding at most
+#endif
+constexpr uint64_t WAIT_LIMIT_NS = 1000000000ull;   // one second per wait
+constexpr uint32_t EP_HEADER_WORDS = 64;             // word 0 = abort flag
+
+struct EpochArgs {
+    const float *y;
+    uint64_t y_stride;
+    uint64_t n_local;       // rows per worker
+    uint64_t d;
+    uint32_t K, batch, nsteps;
+    uint32_t m_last;        // rows of the last minibatch
+    uint32_t nsub_max, nsub_last;
+    uint32_t cols;          // columns per CTA, multiple of 4
+    uint32_t gpad;          // CTA count rounded up to a multiple of 32
+    float lr;
+    float *u;
+    uint64_t u_stride;
+    uint32_t *header;       // [0] abort flag
+    uint32_t *counters;     // one per tile, zero at launch
+    float *partial;         // [EP_RING][batch][gpad], columns >= gridDim.x stay zero
+    uint32_t *status;
+};
+
+// ------------------------------------------------------------- primitives ----
+__device__ __forceinline__ uint32_t smem_u32(const void *p)
+{
+    return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ uint64_t now_ns()
+{
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0u;
+}
+// Bounded wait for phase `parity` of a barrier; gives up early when `*stop` is set.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const volatile uint32_t *stop)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const uint64_t t0 = now_ns();
+    for (;;) {
+        for (int n = 0; n < 32; ++n)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*stop != 0u || now_ns() - t0 > WAIT_LIMIT_NS) return false;
+    }
+}
+// One 2-D box of the row-major matrix X: columns [x, x + box width), rows [y, y + SUB).
+// x * 4 bytes is a multiple of 16; dst is 128-byte aligned.  No multicast.
+__device__ __forceinline__ void tma_load_box(float *dst, const CUtensorMap *map, uint32_t x, uint32_t y,
+                                             uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::
+            "r"(smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+__device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Sum over the 32 lanes of 8 per-lane values at once: three halving exchanges leave one
+// value per lane, two plain butterflies finish.  Lane L ends with the total of value
+// 4*bit4(L) + 2*bit3(L) + bit2(L); the order of the additions is fixed.
+__device__ __forceinline__ float reduce8(float (&v)[8], uint32_t lane)
+{
+    const bool h4 = lane & 16u, h3 = lane & 8u, h2 = lane & 4u;
+    float a[4], b[2];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const float keep = h4 ? v[r + 4] : v[r], send = h4 ? v[r] : v[r + 4];
+        a[r] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 16);
+    }
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const float keep = h3 ? a[r + 2] : a[r], send = h3 ? a[r] : a[r + 2];
+        b[r] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 8);
+    }
+    const float keep = h2 ? b[1] : b[0], send = h2 ? b[0] : b[1];
+    float c = keep + __shfl_xor_sync(0xFFFFFFFFu, send, 4);
+    c += __shfl_xor_sync(0xFFFFFFFFu, c, 2);
+    c += __shfl_xor_sync(0xFFFFFFFFu, c, 1);
+    return c;
+}
+__device__ __forceinline__ uint32_t reduce8_row(uint32_t lane)
+{
+    return ((lane >> 4) & 1u) * 4u + ((lane >> 3) & 1u) * 2u + ((lane >> 2) & 1u);
+}
+
+struct Tile {
+    uint32_t t, k, m, nsub;
+};
+__device__ __forceinline__ Tile tile_of(const EpochArgs &a, uint32_t i)
+{
+    Tile r;
+    r.t = i / a.K;
+    r.k = i - r.t * a.K;
+    const bool last = r.t == a.nsteps - 1u;
+    r.m = last ? a.m_last : a.batch;
+    r.nsub = last ? a.nsub_last : a.nsub_max;
+    return r;
+}
+
+extern __shared__ __align__(1024) unsigned char ep_smem[];
+
+// Shared memory: two tile buffers of nsub_max slots of SUB x cols floats (a slot holds
+// the box of the first 256 columns, then the box of the rest), the step coefficients of
+// the two consumer groups, the barriers, a few flag words.
+__global__ void __launch_bounds__(EP_THREADS, 1)
+    qesgd_lr_epoch_kernel(const EpochArgs a, const __grid_constant__ CUtensorMap map_a,
+                          const __grid_constant__ CUtensorMap map_b)
+{
+    const uint32_t slot_floats = SUB * a.cols;
+    float *const tile = reinterpret_cast<float *>(ep_smem);
+    float *const s_coef = tile + (size_t)2u * a.nsub_max * slot_floats;
+    uint64_t *const full = reinterpret_cast<uint64_t *>(s_coef + 2 * EP_MAX_M);
+    uint64_t *const consumed = full + 2 * EP_MAX_NSUB;
+    // [0] a wait ran out in this CTA, [1] tiles the producer has requested, [2] producer has
+    // stopped, [3] always zero, [4], [5] tiles completed by consumer group 0, 1
+    volatile uint32_t *const s_flag = reinterpret_cast<volatile uint32_t *>(consumed + 2);
+
+    const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
+    const uint32_t cta = blockIdx.x, ncta = gridDim.x;
+    const uint32_t c0 = cta * a.cols;
+    const uint32_t cols_a = min(a.cols, (uint32_t)EP_BOX_COLS), cols_b = a.cols - cols_a;
+    const uint32_t ntiles = a.nsteps * a.K;
+
+    if (tid == 0) {
+        for (uint32_t s = 0; s < 2u * a.nsub_max; ++s) mbar_init(&full[s], 1u);
+        mbar_init(&consumed[0], 1u);
+        mbar_init(&consumed[1], 1u);
+        for (int f = 0; f < 8; ++f) s_flag[f] = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+
+    // ------------------------------------------------------------ producer ----
+    if (warp == EP_CONSUMERS / 32) {
+        for (uint32_t i = 0; i < ntiles; ++i) {
+            const uint32_t b = i & 1u;
+            if (i >= 2u) {   // the buffer is free once the update of tile i-2 has read it
+                const bool ok =
+                    __all_sync(0xFFFFFFFFu, mbar_wait(&consumed[b], ((i - 2u) >> 1) & 1u, &s_flag[0])) != 0;
+                if (!ok) {
+                    if (lane == 0) {
+                        s_flag[0] = 1u;
+                        atomicOr(a.status, QESGD_STATUS_TIMEOUT);
+                        atomicExch(a.header, 1u);
+                    }
+                    break;
+                }
+            }
+            const Tile T = tile_of(a, i);
+            const uint32_t row0 = (uint32_t)((uint64_t)T.k * a.n_local + (uint64_t)T.t * a.batch);
+            // Sub-tiles are requested in order with at most EP_INFLIGHT of them outstanding:
+            // an ordinary load or fence of this SM queues behind the copies already
+            // requested, so a whole tile requested at once would add its transfer time to
+            // every round trip of the consumer warps.
+            bool paced = true;
+            for (uint32_t s = 0; s < T.nsub && paced; ++s) {
+                if (s >= (uint32_t)EP_INFLIGHT) {
+                    paced = __all_sync(0xFFFFFFFFu, mbar_wait(&full[b * a.nsub_max + s - EP_INFLIGHT],
+                                                              (i >> 1) & 1u, &s_flag[0])) != 0;
+                } else if (i > 0u) {
+                    const Tile P = tile_of(a, i - 1u);
+                    if (P.nsub + s >= (uint32_t)EP_INFLIGHT)
+                        paced = __all_sync(0xFFFFFFFFu,
+                                           mbar_wait(&full[(b ^ 1u) * a.nsub_max + P.nsub + s - EP_INFLIGHT],
+                                                     ((i - 1u) >> 1) & 1u, &s_flag[0])) != 0;
+                }
+                if (paced && lane == 0) {
+                    uint64_t *const bar = &full[b * a.nsub_max + s];
+                    float *const dst = tile + (size_t)(b * a.nsub_max + s) * slot_floats;
+                    mbar_arrive_expect_tx(bar, slot_floats * 4u);
+                    tma_load_box(dst, &map_a, c0, row0 + s * SUB, bar);
+                    if (cols_b) tma_load_box(dst + SUB * cols_a, &map_b, c0 + cols_a, row0 + s * SUB, bar);
+                }
+            }
+            if (!paced) {
+                if (lane == 0) {
+                    s_flag[0] = 1u;
+                    atomicOr(a.status, QESGD_STATUS_TIMEOUT);
+                    atomicExch(a.header, 1u);
+                }
+                break;
+            }
+            __syncwarp();
+            if (lane == 0) s_flag[1] = i + 1u;
+        }
+        __syncwarp();
+        if (lane == 0) {
+            __threadfence_block();
+            s_flag[2] = 1u;
+        }
+        return;
+    }
+
+    // ----------------------------------------------------------- consumers ----
+    // Two groups of four warps; group g owns buffer g and the tiles i = g, g+2, g+4, ...
+    // Each runs M(i), W(i), U(i) for its own tiles, so that one group computes while the
+    // other waits for the other CTAs.
+    const uint32_t g = warp >> 2, wg = warp & 3u, tg = tid & (EP_GROUP - 1u);
+    float *const coef = s_coef + g * EP_MAX_M;
+    auto group_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(1u + g), "n"(EP_GROUP) : "memory"); };
+
+    for (uint32_t i = g; i < ntiles; i += 2u) {
+        const Tile T = tile_of(a, i);
+        const uint32_t parity = (i >> 1) & 1u;
+        uint64_t *const bars = full + g * a.nsub_max;
+        const float *const buf = tile + (size_t)g * a.nsub_max * slot_floats;
+
+        // The worker's previous minibatch is tile i-K.  With an odd K it belonged to the other
+        // group: wait until that group has stored its update.
+        if (i >= a.K && ((i - a.K) & 1u) != g) {
+            const uint32_t need = ((i - a.K) >> 1) + 1u;
+            if (tg == 0) {
+                const uint64_t t0 = now_ns();
+                while (s_flag[4u + (g ^ 1u)] < need) {
+                    if (s_flag[0] != 0u || now_ns() - t0 > WAIT_LIMIT_NS) {
+                        s_flag[0] = 1u;
+                        break;
+                    }
+                }
+                __threadfence_block();
+            }
+            group_sync();
+            if (s_flag[0] != 0u) break;
+        }
+
+        // ---- M(i): margins over this CTA's columns, then the signal to the other CTAs ----
+        {
+            const float *__restrict__ ug = a.u + (uint64_t)T.k * a.u_stride + c0;
+            float4 uu[EP_MAX_COLS / 128];
+#pragma unroll
+            for (int it = 0; it < EP_MAX_COLS / 128; ++it) {
+                const uint32_t c = lane * 4u + it * 128u;
+                uu[it] = (c < a.cols && (uint64_t)c0 + c < a.d) ? *reinterpret_cast<const float4 *>(ug + c)
+                                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            float *__restrict__ pout = a.partial + ((uint64_t)(i % EP_RING) * a.batch) * a.gpad + cta;
+            bool ok = true;
+            for (uint32_t s = wg; s < T.nsub; s += EP_GROUP / 32) {   // a warp per sub-tile
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars[s], parity, &s_flag[0])) != 0;
+                if (!ok) break;
+                const float *__restrict__ xs = buf + (size_t)s * slot_floats;
+                float acc[SUB];
+#pragma unroll
+                for (int r = 0; r < SUB; ++r) acc[r] = 0.0f;
+#pragma unroll
+                for (int it = 0; it < EP_MAX_COLS / 128; ++it) {
+                    const uint32_t c = lane * 4u + it * 128u;
+                    if (c < a.cols) {
+                        const bool first = it < EP_BOX_COLS / 128;
+                        const float *__restrict__ base = first ? xs + c : xs + SUB * cols_a + (c - EP_BOX_COLS);
+                        const uint32_t pitch = first ? cols_a : cols_b;
+#pragma unroll
+                        for (int r = 0; r < SUB; ++r) {
+                            const float4 x = *reinterpret_cast<const float4 *>(base + r * pitch);
+                            acc[r] = fmaf(x.x, uu[it].x, acc[r]);
+                            acc[r] = fmaf(x.y, uu[it].y, acc[r]);
+                            acc[r] = fmaf(x.z, uu[it].z, acc[r]);
+                            acc[r] = fmaf(x.w, uu[it].w, acc[r]);
+                        }
+                    }
+                }
+                const float tot = reduce8(acc, lane);
+                const uint32_t jj = s * SUB + reduce8_row(lane);
+                if ((lane & 3u) == 0u && jj < T.m) pout[(uint64_t)jj * a.gpad] = tot;
+            }
+            if (!ok) s_flag[0] = 1u;
+            group_sync();
+            if (s_flag[0] != 0u) break;
+            if (tg == 0) {
+                asm volatile("fence.acq_rel.gpu;" ::: "memory");   // partials before the count
+                atomicAdd(a.counters + i, 1u);
+            }
+        }
+
+        // ---- W(i): all CTAs' partial margins -> step coefficients in shared memory ----
+        {
+            // the labels of the rows this lane will finish, requested before the wait
+            const float *__restrict__ yt = a.y + (uint64_t)T.k * a.y_stride + (uint64_t)T.t * a.batch;
+            if (tg == 0) {
+                const uint64_t t0 = now_ns();
+                uint32_t n = 0u;
+                while (ld_acquire(a.counters + i) < ncta) {
+                    if ((++n & 31u) == 0u) {
+                        if (s_flag[0] != 0u || ld_acquire(a.header) != 0u || now_ns() - t0 > WAIT_LIMIT_NS) {
+                            s_flag[0] = 1u;
+                            break;
+                        }
+                        __nanosleep(64);
+                    }
+                }
+            }
+            group_sync();
+            if (s_flag[0] != 0u) break;
+            // a warp sums eight rows at a time: lanes along the CTA index (contiguous in memory)
+            const float *__restrict__ pin = a.partial + ((uint64_t)(i % EP_RING) * a.batch) * a.gpad;
+            for (uint32_t j0 = wg * SUB; j0 < T.m; j0 += EP_GROUP / 32 * SUB) {
+                const uint32_t j = j0 + reduce8_row(lane);
+                const float yj = j < T.m ? __ldg(yt + j) : 0.0f;
+                // all sixteen loads of a lane are requested before the first is used (gpad <= 256)
+                float4 q0[SUB], q1[SUB];
+#pragma unroll
+                for (int r = 0; r < SUB; ++r) {
+                    const float *__restrict__ p = pin + (uint64_t)min(j0 + r, T.m - 1u) * a.gpad;
+                    q0[r] = q1[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (lane * 4u < a.gpad) q0[r] = __ldcg(reinterpret_cast<const float4 *>(p + lane * 4u));
+                    if (128u + lane * 4u < a.gpad)
+                        q1[r] = __ldcg(reinterpret_cast<const float4 *>(p + 128u + lane * 4u));
+                }
+                float v[SUB];
+#pragma unroll
+                for (int r = 0; r < SUB; ++r)
+                    v[r] = ((q0[r].x + q0[r].y) + (q0[r].z + q0[r].w)) +
+                           ((q1[r].x + q1[r].y) + (q1[r].z + q1[r].w));
+                const float margin = reduce8(v, lane);
+                // -(lr/m) * c_j with c_j = -y_j / (1 + exp(y_j m_j))
+                if ((lane & 3u) == 0u && j < T.m)
+                    coef[j] = (a.lr / (float)T.m) * yj / (1.0f + expf(yj * margin));
+            }
+            group_sync();
+        }
+
+        // ---- U(i): update this CTA's columns of u from the buffer, release the buffer ----
+        {
+            const uint32_t col = tg * 4u;
+            const bool colok = col < a.cols && (uint64_t)c0 + col < a.d;
+            const bool first = col < (uint32_t)EP_BOX_COLS;
+            const uint32_t off = first ? col : SUB * cols_a + (col - EP_BOX_COLS);
+            const uint32_t pitch = first ? cols_a : cols_b;
+            float4 *const up = reinterpret_cast<float4 *>(a.u + (uint64_t)T.k * a.u_stride + c0 + col);
+            float4 uold = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (colok) uold = *up;                       // requested now, needed after the loop
+            // every thread observes the arrivals itself before it reads what TMA wrote
+            for (uint32_t s = 0; s < T.nsub; ++s) mbar_wait(&bars[s], parity, &s_flag[0]);
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (colok) {
+                for (uint32_t s = 0; s < T.nsub; ++s) {
+                    const float *__restrict__ base = buf + (size_t)s * slot_floats + off;
+#pragma unroll
+                    for (uint32_t r = 0; r < (uint32_t)SUB; ++r) {
+                        const uint32_t jj = s * SUB + r;
+                        if (jj < T.m) {
+                            const float4 x = *reinterpret_cast<const float4 *>(base + (size_t)r * pitch);
+                            const float cj = coef[jj];
+                            acc.x = fmaf(cj, x.x, acc.x);
+                            acc.y = fmaf(cj, x.y, acc.y);
+                            acc.z = fmaf(cj, x.z, acc.z);
+                            acc.w = fmaf(cj, x.w, acc.w);
+                        }
+                    }
+                }
+                uold.x += acc.x;
+                uold.y += acc.y;
+                uold.z += acc.z;
+                uold.w += acc.w;
+                *up = uold;
+            }
+            group_sync();                                 // buffer read, u stored, by the whole group
+            if (tg == 0) {
+                mbar_arrive(&consumed[g]);                // hand the buffer back to the producer
+                __threadfence_block();
+                s_flag[4u + g] = (i >> 1) + 1u;           // this group's tiles completed
+            }
+        }
+    }
+
+    // Both groups meet here, whether they finished or gave up.
+    asm volatile("bar.sync 3, %0;" ::"n"(EP_CONSUMERS) : "memory");
+    if (s_flag[0] == 0u) return;
+
+    // ---- a wait ran out: tell the others, let the copies in flight land, leave --------
+    if (tid == 0) {
+        atomicOr(a.status, QESGD_STATUS_TIMEOUT);
+        atomicExch(a.header, 1u);
+    }
+    {
+        const uint64_t t0 = now_ns();
+        while (s_flag[2] == 0u && now_ns() - t0 < 2u * WAIT_LIMIT_NS) __nanosleep(256);
+    }
+    const uint32_t issued = s_flag[1];
+    for (uint32_t b = 0; b < 2u && b < issued; ++b) {
+        const uint32_t last = ((issued - 1u - b) & ~1u) + b;   // last requested tile of buffer b
+        const Tile T = tile_of(a, last);
+        for (uint32_t s = 0; s < T.nsub; ++s)
+            if (!mbar_wait(&full[b * a.nsub_max + s], (last >> 1) & 1u, &s_flag[3])) return;
+    }
+}
+
+// ------------------------------------------------------------------ host ----
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+// Per-device set-up: shared-memory limit of the kernel, the driver's tensor-map encoder.
+constexpr int MAX_DEVICES = 64;
+std::mutex g_epoch_mutex;
+int g_epoch_smem_limit[MAX_DEVICES] = {0};   // 0 = not queried, -1 = unsupported
+EncodeTiledFn g_encode_tiled = nullptr;
+
+int epoch_smem_limit(int device)
+{
+    if (device < 0 || device >= MAX_DEVICES) return -1;
+    std::lock_guard<std::mutex> lock(g_epoch_mutex);
+    if (g_epoch_smem_limit[device] == 0) {
+        int coop = 0, optin = 0;
+        cudaError_t e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device);
+        if (e == cudaSuccess)
+            e = cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device);
+        if (e == cudaSuccess && coop && optin > 0)
+            e = cudaFuncSetAttribute(qesgd_lr_epoch_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     optin);
+        if (e == cudaSuccess && !g_encode_tiled) {
+            void *fn = nullptr;
+            cudaDriverEntryPointQueryResult q = cudaDriverEntryPointSymbolNotFound;
+            e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+            if (e == cudaSuccess && q == cudaDriverEntryPointSuccess) g_encode_tiled = (EncodeTiledFn)fn;
+        }
+        g_epoch_smem_limit[device] =
+            (e == cudaSuccess && coop && optin > 0 && g_encode_tiled) ? optin : -1;
+        if (e != cudaSuccess) cudaGetLastError();
+    }
+    return g_epoch_smem_limit[device];
+}
+
+// Row-major float matrix [rows][d] seen as a 2-D tensor; a box is SUB rows of box_cols columns.
+// Elements outside the matrix read as zero.
+bool make_map(CUtensorMap *map, const float *X, uint64_t rows, uint64_t d, uint32_t box_cols)
+{
+    const cuuint64_t dims[2] = {d, rows};
+    const cuuint64_t strides[1] = {d * sizeof(float)};
+    const cuuint32_t box[2] = {box_cols, (cuuint32_t)SUB};
+    const cuuint32_t elem[2] = {1u, 1u};
+    return g_encode_tiled(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2u, const_cast<float *>(X), dims, strides, box,
+                          elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+// Returns 0 = launched, -1 = shape not covered by the fused kernel (caller uses the
+// two-pass steps), > 0 = cudaError_t.
+int qesgd_launch_lr_epoch_fused(const float *X, const float *y, uint64_t n_local, uint64_t d,
+                                uint32_t K, uint32_t batch, float lr, float *u, uint64_t u_stride,
+                                float *work, uint64_t work_floats, uint32_t *status, int device,
+                                int sm_count, cudaStream_t stream, int *launched)
+{
+    *launched = 0;
+    const uint32_t m_full = (uint32_t)(n_local < batch ? n_local : batch);
+    if (m_full > (uint32_t)EP_MAX_M) return -1;
+    const uint64_t nsteps64 = (n_local + m_full - 1) / m_full;
+    if (nsteps64 * K > (1u << 20)) return -1;
+    if ((uint64_t)K * n_local + EP_MAX_M >= (1ull << 31)) return -1;   // TMA row coordinates
+    if (d % 4 != 0 || u_stride % 4 != 0 || ((uintptr_t)X | (uintptr_t)u) % 16 != 0) return -1;
+    if (sm_count < 1) return -1;
+    uint64_t cols = (d + (uint64_t)sm_count - 1) / (uint64_t)sm_count;
+    cols = (cols + 3) / 4 * 4;
+    if (cols > (uint64_t)EP_MAX_COLS) return -1;
+    const uint32_t ncta = (uint32_t)((d + cols - 1) / cols);
+    if (ncta > 256u) return -1;   // a lane sums at most two groups of four CTAs per row
+    const int limit = epoch_smem_limit(device);
+    if (limit <= 0) return -1;
+
+    EpochArgs a;
+    a.y = y; a.y_stride = n_local; a.n_local = n_local;
+    a.d = d; a.K = K; a.batch = m_full; a.nsteps = (uint32_t)nsteps64;
+    a.m_last = (uint32_t)(n_local - (nsteps64 - 1) * m_full);
+    a.nsub_max = (m_full + SUB - 1) / SUB;
+    a.nsub_last = (a.m_last + SUB - 1) / SUB;
+    a.cols = (uint32_t)cols;
+    a.gpad = (ncta + 31u) / 32u * 32u;
+    a.lr = lr;
+    a.u = u; a.u_stride = u_stride;
+    a.status = status;
+
+    // shared memory: two tile buffers | coefficients of both groups | barriers | flags
+    const size_t smem = (size_t)2 * a.nsub_max * SUB * cols * sizeof(float) + 2 * EP_MAX_M * sizeof(float) +
+                        (2 * EP_MAX_NSUB + 2) * sizeof(uint64_t) + 32;
+    if (smem > (size_t)limit) return -1;
+
+    // workspace: header | one counter per tile | partial margins
+    const uint64_t ntiles = nsteps64 * K;
+    const uint64_t counter_words = (ntiles + 63) / 64 * 64;
+    const uint64_t partial_floats = (uint64_t)EP_RING * m_full * a.gpad;
+    const uint64_t words = EP_HEADER_WORDS + counter_words + partial_floats;
+    if (words > work_floats) return -1;
+    a.header = reinterpret_cast<uint32_t *>(work);
+    a.counters = a.header + EP_HEADER_WORDS;
+    a.partial = work + EP_HEADER_WORDS + counter_words;
+
+    CUtensorMap map_a, map_b;
+    const uint32_t cols_a = cols < (uint64_t)EP_BOX_COLS ? (uint32_t)cols : (uint32_t)EP_BOX_COLS;
+    const uint32_t cols_b = (uint32_t)cols - cols_a;
+    if (!make_map(&map_a, X, (uint64_t)K * n_local, d, cols_a)) return -1;
+    if (!make_map(&map_b, X, (uint64_t)K * n_local, d, cols_b ? cols_b : cols_a)) return -1;
+
+    cudaError_t e = cudaMemsetAsync(work, 0, words * sizeof(float), stream);
+    if (e != cudaSuccess) return (int)e;
+    void *params[] = {(void *)&a, (void *)&map_a, (void *)&map_b};
+    e = cudaLaunchCooperativeKernel((const void *)qesgd_lr_epoch_kernel, dim3(ncta), dim3(EP_THREADS), params,
+                                    smem, stream);
+    if (e != cudaSuccess) return (int)e;
+    *launched = 1;
+    return 0;
+}

@@ -12,6 +12,7 @@ LIB_PATH = os.path.join(_HERE, "libqesgd.so")
 
 SCALE_NORM, SCALE_MAX, SCALE_FIXED = 0, 1, 2
 STATUS_NONFINITE = 1
+STATUS_TIMEOUT = 2
 OK, EINVAL, ECUDA, ENOMEM, ELIMIT = 0, -1, -2, -3, -4
 MAX_WORKERS, MIN_BUCKET, MAX_BUCKET, MAX_LR_BATCH = 64, 64, 8192, 1024
 NOALLOC_MAX_LR_BATCH = 256

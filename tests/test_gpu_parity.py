@@ -323,6 +323,41 @@ def test_lr_local_epoch_and_batch_match_oracle():
     assert (t1.cpu().numpy() == got[0]).all()
 
 
+@pytest.mark.parametrize("K,n_local,d,batch", [
+    (1, 130, 4096, 64),      # one worker: every minibatch waits for the previous update
+    (2, 128, 8192, 64),      # even K: a worker's minibatches stay in one consumer group
+    (4, 96, 65536, 32),      # the benchmark's width (444 columns per CTA, two TMA boxes)
+    (5, 77, 1000, 20),       # odd K, rows not a multiple of 8, ragged last minibatch of 17
+    (3, 300, 2048, 256),     # the largest minibatch the persistent kernel takes
+    (2, 40, 75776, 8),       # the widest slice (512 columns per CTA)
+    (2, 600, 1024, 300),     # minibatch above 256 rows: two-pass steps
+    (2, 64, 1002, 32),       # d not a multiple of 4: two-pass steps
+    (2, 64, 80000, 32),      # d above 512 columns per SM: two-pass steps
+])
+def test_lr_local_epoch_shapes_match_oracle(K, n_local, d, batch):
+    """The local epoch through the C ABI against the fp64 oracle, over shapes that take the
+    persistent kernel (shared-memory tiles, inter-CTA margins) and shapes that fall back to
+    one margin pass and one update pass per minibatch."""
+    X, y, _ = synthetic.logistic_problem(K * n_local, d, seed=K + n_local + d)
+    u0 = (0.1 * synthetic.normal_f32(d, 1.0, 21)).astype(np.float32)
+    stride = d + 4 * (K % 2)                       # padded rows for odd K
+    tu = torch.zeros((K, stride), dtype=torch.float32, device="cuda")
+    tu[:, :d] = G.dev(u0)
+    c = G.ctx()
+    c.qesgd_lr_local_epoch_batch(G.dev(X), G.dev(y), n_local, d, K, batch, 0.5, tu, stride)
+    assert c.qesgd_status() == 0
+    got = tu.cpu().numpy()
+    for k in range(K):
+        rows = slice(k * n_local, (k + 1) * n_local)
+        _lr_close(got[k, :d], ref.lr_local_epoch(X[rows], y[rows], batch, 0.5, u0))
+    assert (got[:, d:] == 0).all()
+    # the same call again gives the same bits (fixed summation order, no atomics on data)
+    tu2 = torch.zeros((K, stride), dtype=torch.float32, device="cuda")
+    tu2[:, :d] = G.dev(u0)
+    c.qesgd_lr_local_epoch_batch(G.dev(X), G.dev(y), n_local, d, K, batch, 0.5, tu2, stride)
+    assert torch.equal(tu, tu2)
+
+
 # ----------------------------------------------- per-step QESGD (Algorithm 2) ---
 def _gpu_requantize(u, w, zsum, bucket, s, bits, mode, seed, worker, step, fixed_delta=0.0,
                     misalign=0):
