@@ -48,9 +48,6 @@ constexpr int EP_MAX_COLS = 512;     // columns per CTA: 128 groups of 4
 constexpr int EP_BOX_COLS = 256;     // widest TMA box
 constexpr int EP_MAX_M = 256;        // rows per minibatch the fused path takes
 constexpr int EP_MAX_NSUB = EP_MAX_M / SUB;
-#ifndef EP_INFLIGHT
-#define EP_INFLIGHT 3               // sub-tiles a CTA has outstanding at most
-#endif
 constexpr uint64_t WAIT_LIMIT_NS = 1000000000ull;   // one second per wait
 constexpr uint32_t EP_HEADER_WORDS = 64;             // word 0 = abort flag
 
@@ -199,7 +196,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
     uint64_t *const consumed = full + 2 * EP_MAX_NSUB;
     // [0] a wait ran out in this CTA, [1] tiles the producer has requested, [2] producer has
     // stopped, [3] always zero, [4], [5] tiles completed by consumer group 0, 1
-    volatile uint32_t *const s_flag = reinterpret_cast<volatile uint32_t *>(consumed + 2);
+    volatile uint32_t *const s_flag = reinterpret_cast<volatile uint32_t *>(consumed + 2 * EP_MAX_NSUB);
 
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
     const uint32_t cta = blockIdx.x, ncta = gridDim.x;
@@ -209,8 +206,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
 
     if (tid == 0) {
         for (uint32_t s = 0; s < 2u * a.nsub_max; ++s) mbar_init(&full[s], 1u);
-        mbar_init(&consumed[0], 1u);
-        mbar_init(&consumed[1], 1u);
+        for (uint32_t s = 0; s < 2u * a.nsub_max; ++s) mbar_init(&consumed[s], EP_GROUP / 32);
         for (int f = 0; f < 8; ++f) s_flag[f] = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -220,37 +216,15 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
     if (warp == EP_CONSUMERS / 32) {
         for (uint32_t i = 0; i < ntiles; ++i) {
             const uint32_t b = i & 1u;
-            if (i >= 2u) {   // the buffer is free once the update of tile i-2 has read it
-                const bool ok =
-                    __all_sync(0xFFFFFFFFu, mbar_wait(&consumed[b], ((i - 2u) >> 1) & 1u, &s_flag[0])) != 0;
-                if (!ok) {
-                    if (lane == 0) {
-                        s_flag[0] = 1u;
-                        atomicOr(a.status, QESGD_STATUS_TIMEOUT);
-                        atomicExch(a.header, 1u);
-                    }
-                    break;
-                }
-            }
             const Tile T = tile_of(a, i);
             const uint32_t row0 = (uint32_t)((uint64_t)T.k * a.n_local + (uint64_t)T.t * a.batch);
-            // Sub-tiles are requested in order with at most EP_INFLIGHT of them outstanding:
-            // an ordinary load or fence of this SM queues behind the copies already
-            // requested, so a whole tile requested at once would add its transfer time to
-            // every round trip of the consumer warps.
-            bool paced = true;
-            for (uint32_t s = 0; s < T.nsub && paced; ++s) {
-                if (s >= (uint32_t)EP_INFLIGHT) {
-                    paced = __all_sync(0xFFFFFFFFu, mbar_wait(&full[b * a.nsub_max + s - EP_INFLIGHT],
-                                                              (i >> 1) & 1u, &s_flag[0])) != 0;
-                } else if (i > 0u) {
-                    const Tile P = tile_of(a, i - 1u);
-                    if (P.nsub + s >= (uint32_t)EP_INFLIGHT)
-                        paced = __all_sync(0xFFFFFFFFu,
-                                           mbar_wait(&full[(b ^ 1u) * a.nsub_max + P.nsub + s - EP_INFLIGHT],
-                                                     ((i - 1u) >> 1) & 1u, &s_flag[0])) != 0;
-                }
-                if (paced && lane == 0) {
+            bool ok = true;
+            for (uint32_t s = 0; s < T.nsub && ok; ++s) {
+                // a slot is free once the update of tile i-2 has read sub-tile s
+                if (i >= 2u)
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(&consumed[b * a.nsub_max + s],
+                                                           ((i - 2u) >> 1) & 1u, &s_flag[0])) != 0;
+                if (ok && lane == 0) {
                     uint64_t *const bar = &full[b * a.nsub_max + s];
                     float *const dst = tile + (size_t)(b * a.nsub_max + s) * slot_floats;
                     mbar_arrive_expect_tx(bar, slot_floats * 4u);
@@ -258,7 +232,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
                     if (cols_b) tma_load_box(dst + SUB * cols_a, &map_b, c0 + cols_a, row0 + s * SUB, bar);
                 }
             }
-            if (!paced) {
+            if (!ok) {
                 if (lane == 0) {
                     s_flag[0] = 1u;
                     atomicOr(a.status, QESGD_STATUS_TIMEOUT);
@@ -284,6 +258,22 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
     const uint32_t g = warp >> 2, wg = warp & 3u, tg = tid & (EP_GROUP - 1u);
     float *const coef = s_coef + g * EP_MAX_M;
     auto group_sync = [&]() { asm volatile("bar.sync %0, %1;" ::"r"(1u + g), "n"(EP_GROUP) : "memory"); };
+
+    // this lane's columns of worker k's u (columns lane*4 + 128*it), zeros past the slice
+    auto load_u = [&](uint32_t k, float4 (&uu)[EP_MAX_COLS / 128]) {
+        const float *__restrict__ ug = a.u + (uint64_t)k * a.u_stride + c0;
+#pragma unroll
+        for (int it = 0; it < EP_MAX_COLS / 128; ++it) {
+            const uint32_t c = lane * 4u + it * 128u;
+            uu[it] = (c < a.cols && (uint64_t)c0 + c < a.d) ? *reinterpret_cast<const float4 *>(ug + c)
+                                                           : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+    // With an even K >= 4 the group's next tile belongs to a worker whose previous minibatch
+    // this group finished an iteration ago: its slice of u is requested a tile early.
+    const bool early_u = (a.K & 1u) == 0u && a.K >= 4u;
+    float4 un[EP_MAX_COLS / 128];
+    if (early_u && g < ntiles) load_u(g % a.K, un);
 
     for (uint32_t i = g; i < ntiles; i += 2u) {
         const Tile T = tile_of(a, i);
@@ -311,13 +301,13 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
 
         // ---- M(i): margins over this CTA's columns, then the signal to the other CTAs ----
         {
-            const float *__restrict__ ug = a.u + (uint64_t)T.k * a.u_stride + c0;
             float4 uu[EP_MAX_COLS / 128];
+            if (early_u) {
 #pragma unroll
-            for (int it = 0; it < EP_MAX_COLS / 128; ++it) {
-                const uint32_t c = lane * 4u + it * 128u;
-                uu[it] = (c < a.cols && (uint64_t)c0 + c < a.d) ? *reinterpret_cast<const float4 *>(ug + c)
-                                                               : make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int it = 0; it < EP_MAX_COLS / 128; ++it) uu[it] = un[it];
+                if (i + 2u < ntiles) load_u((i + 2u) % a.K, un);
+            } else {
+                load_u(T.k, uu);
             }
             float *__restrict__ pout = a.partial + ((uint64_t)(i % EP_RING) * a.batch) * a.gpad + cta;
             bool ok = true;
@@ -379,28 +369,38 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
             if (s_flag[0] != 0u) break;
             // a warp sums eight rows at a time: lanes along the CTA index (contiguous in memory)
             const float *__restrict__ pin = a.partial + ((uint64_t)(i % EP_RING) * a.batch) * a.gpad;
-            for (uint32_t j0 = wg * SUB; j0 < T.m; j0 += EP_GROUP / 32 * SUB) {
-                const uint32_t j = j0 + reduce8_row(lane);
-                const float yj = j < T.m ? __ldg(yt + j) : 0.0f;
-                // all sixteen loads of a lane are requested before the first is used (gpad <= 256)
-                float4 q0[SUB], q1[SUB];
+            // Two passes of eight rows per iteration; all 32 loads of a lane are requested
+            // before the first is used (gpad <= 256).
+            for (uint32_t j0 = wg * SUB; j0 < T.m; j0 += 2u * (EP_GROUP / 32) * SUB) {
+                float4 q0[2][SUB], q1[2][SUB];
+                float yj[2];
+                uint32_t jrow[2];
 #pragma unroll
-                for (int r = 0; r < SUB; ++r) {
-                    const float *__restrict__ p = pin + (uint64_t)min(j0 + r, T.m - 1u) * a.gpad;
-                    q0[r] = q1[r] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (lane * 4u < a.gpad) q0[r] = __ldcg(reinterpret_cast<const float4 *>(p + lane * 4u));
-                    if (128u + lane * 4u < a.gpad)
-                        q1[r] = __ldcg(reinterpret_cast<const float4 *>(p + 128u + lane * 4u));
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t jh = j0 + h * (EP_GROUP / 32) * SUB;
+                    jrow[h] = jh + reduce8_row(lane);
+                    yj[h] = jrow[h] < T.m ? __ldg(yt + jrow[h]) : 0.0f;
+#pragma unroll
+                    for (int r = 0; r < SUB; ++r) {
+                        const float *__restrict__ p = pin + (uint64_t)min(jh + r, T.m - 1u) * a.gpad;
+                        q0[h][r] = q1[h][r] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        if (lane * 4u < a.gpad) q0[h][r] = __ldcg(reinterpret_cast<const float4 *>(p + lane * 4u));
+                        if (128u + lane * 4u < a.gpad)
+                            q1[h][r] = __ldcg(reinterpret_cast<const float4 *>(p + 128u + lane * 4u));
+                    }
                 }
-                float v[SUB];
 #pragma unroll
-                for (int r = 0; r < SUB; ++r)
-                    v[r] = ((q0[r].x + q0[r].y) + (q0[r].z + q0[r].w)) +
-                           ((q1[r].x + q1[r].y) + (q1[r].z + q1[r].w));
-                const float margin = reduce8(v, lane);
-                // -(lr/m) * c_j with c_j = -y_j / (1 + exp(y_j m_j))
-                if ((lane & 3u) == 0u && j < T.m)
-                    coef[j] = (a.lr / (float)T.m) * yj / (1.0f + expf(yj * margin));
+                for (int h = 0; h < 2; ++h) {
+                    float v[SUB];
+#pragma unroll
+                    for (int r = 0; r < SUB; ++r)
+                        v[r] = ((q0[h][r].x + q0[h][r].y) + (q0[h][r].z + q0[h][r].w)) +
+                               ((q1[h][r].x + q1[h][r].y) + (q1[h][r].z + q1[h][r].w));
+                    const float margin = reduce8(v, lane);
+                    // -(lr/m) * c_j with c_j = -y_j / (1 + exp(y_j m_j))
+                    if ((lane & 3u) == 0u && jrow[h] < T.m)
+                        coef[jrow[h]] = (a.lr / (float)T.m) * yj[h] / (1.0f + expf(yj[h] * margin));
+                }
             }
             group_sync();
         }
@@ -418,8 +418,8 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
             // every thread observes the arrivals itself before it reads what TMA wrote
             for (uint32_t s = 0; s < T.nsub; ++s) mbar_wait(&bars[s], parity, &s_flag[0]);
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (colok) {
-                for (uint32_t s = 0; s < T.nsub; ++s) {
+            for (uint32_t s = 0; s < T.nsub; ++s) {
+                if (colok) {
                     const float *__restrict__ base = buf + (size_t)s * slot_floats + off;
 #pragma unroll
                     for (uint32_t r = 0; r < (uint32_t)SUB; ++r) {
@@ -434,15 +434,20 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
                         }
                     }
                 }
+                // the warp is through with this slot: one arrival per warp hands it back to the
+                // producer, which refills it while the update goes on
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&consumed[g * a.nsub_max + s]);
+            }
+            if (colok) {
                 uold.x += acc.x;
                 uold.y += acc.y;
                 uold.z += acc.z;
                 uold.w += acc.w;
                 *up = uold;
             }
-            group_sync();                                 // buffer read, u stored, by the whole group
+            group_sync();                                 // u stored by the whole group
             if (tg == 0) {
-                mbar_arrive(&consumed[g]);                // hand the buffer back to the producer
                 __threadfence_block();
                 s_flag[4u + g] = (i >> 1) + 1u;           // this group's tiles completed
             }
@@ -561,7 +566,7 @@ int qesgd_launch_lr_epoch_fused(const float *X, const float *y, uint64_t n_local
 
     // shared memory: two tile buffers | coefficients of both groups | barriers | flags
     const size_t smem = (size_t)2 * a.nsub_max * SUB * cols * sizeof(float) + 2 * EP_MAX_M * sizeof(float) +
-                        (2 * EP_MAX_NSUB + 2) * sizeof(uint64_t) + 32;
+                        (4 * EP_MAX_NSUB) * sizeof(uint64_t) + 32;
     if (smem > (size_t)limit) return -1;
 
     // workspace: header | one counter per tile | partial margins
