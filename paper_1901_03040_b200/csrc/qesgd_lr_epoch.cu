@@ -415,8 +415,12 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
             float4 *const up = reinterpret_cast<float4 *>(a.u + (uint64_t)T.k * a.u_stride + c0 + col);
             float4 uold = make_float4(0.f, 0.f, 0.f, 0.f);
             if (colok) uold = *up;                       // requested now, needed after the loop
-            // every thread observes the arrivals itself before it reads what TMA wrote
-            for (uint32_t s = 0; s < T.nsub; ++s) mbar_wait(&bars[s], parity, &s_flag[0]);
+            // Every warp observes the arrival of every sub-tile itself before it reads what TMA
+            // wrote: lane s looks at sub-tile s (a look costs about 0.1 us, so the lanes look in
+            // parallel), and the warp follows its lanes through __syncwarp.  All of them have
+            // landed: the warps that took the margins waited for them.
+            for (uint32_t s = lane; s < T.nsub; s += 32u) mbar_wait(&bars[s], parity, &s_flag[0]);
+            __syncwarp();
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (uint32_t s = 0; s < T.nsub; ++s) {
                 if (colok) {
