@@ -359,7 +359,7 @@ def oracle_sample(ctx, w, locs, stride, anchor, device, sample_elems):
     from oracle import qesgd_ref as ref
     from paper_1901_03040_b200 import qesgd
     d, K, bits, s, B = w["d"], w["K"], w["bits"], w["s"], w["bucket"]
-    n = min(d, sample_elems // B * B)
+    n = min(d, sample_elems) // B * B          # whole buckets only
     nb = n // B
     param = anchor.clone()
     codes, scales = qesgd.alloc_stream_buffers(K, d, B, bits, device)
