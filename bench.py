@@ -592,6 +592,13 @@ def run_c1(args, device, world, rank):
                                    "one local epoch of minibatch-64 SGD (lr 0.1), 8-bit codes, bucket 512"},
             "gpu_launches": int(ctx.qesgd_launch_count() - launches0),
             "kernels": {k: {"avg_ms": statistics.mean(v)} for k, v in times.items()},
+            "roofline": {"bound": "hbm", "kernel": "qesgd_lr_epoch_kernel (local epoch of all workers)",
+                         "achieved": n * d * 4 / (statistics.mean(times["local_epoch"]) * 1e-3) / 1e9,
+                         "peak": peaks()[0], "unit": "GB/s",
+                         "frac": n * d * 4 / (statistics.mean(times["local_epoch"]) * 1e-3) / 1e9 / peaks()[0],
+                         "traffic": None, "peak_source": peaks()[1],
+                         "algorithmic_bytes_per_launch": float(n * d * 4)},
+            "status_flags": ctx.qesgd_status(),
             "x_bytes_per_epoch": int(n * d * 4),
             # algorithmic bytes of the epoch: every row of X once (the minibatch stays on chip
             # between the margin pass and the update pass)
