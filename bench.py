@@ -562,6 +562,7 @@ def run_c1(args, device, world, rank):
     times = {"local_epoch": [], "encode": [], "apply": []}
     launches0 = None
     losses = []
+    first_round = {}
     for it in range(args.warmup + args.steps):
         if it == args.warmup:
             launches0 = ctx.qesgd_launch_count()
@@ -579,6 +580,9 @@ def run_c1(args, device, world, rank):
         e[3].record(stream)
         torch.cuda.synchronize()
         losses.append(loss(param))
+        if it == 0:   # round 1 (from w = 0), outside every timed region
+            first_round = c1_first_round(args, rank, world, X, y, u, codes, scales, param, loss,
+                                         (n_local, d, K, batch, lr, B, s, bits))
         if it >= args.warmup:
             times["local_epoch"].append(e[0].elapsed_time(e[1]))
             times["encode"].append(e[1].elapsed_time(e[2]))
@@ -604,9 +608,52 @@ def run_c1(args, device, world, rank):
             # between the margin pass and the update pass)
             "local_epoch_gbs": n * d * 4 / (statistics.mean(times["local_epoch"]) * 1e-3) / 1e9,
             "loss_before": loss0, "loss_after_first_rounds": losses[:3], "loss_after_last_round": losses[-1],
-            "rounds": len(losses)}
+            "rounds": len(losses), "first_round": first_round}
+    if "oracle" in first_round:
+        o = first_round["oracle"]
+        line["cpu_baseline"] = {"value": 1e3 * (o["oracle_local_epoch_s"] + o["oracle_codec_s"]), "unit": "ms",
+                                "cores": 1, "kind": "oracle",
+                                "sample": "the whole of round 1: four local epochs, encode of the four "
+                                          "workers, decode-average-apply"}
     if rank == 0:
         print(json.dumps(line))
+
+
+def c1_first_round(args, rank, world, X, y, u, codes, scales, param, loss, shape):
+    """Round 1 of C1 looked at from outside the timed region: the loss the unquantised average of
+    the workers' parameters would have given (Sec. 5 claims 8 bits lose nothing against plain
+    SGD), and, with the CPU oracle, the same round on the host: the oracle's local epochs against
+    the GPU's (tolerance), then hand-off parity -- the oracle encodes the GPU's u_k and its codes
+    and scales must equal the GPU's bit for bit, its applied parameter within 1e-6."""
+    import numpy as np
+    import torch
+    n_local, d, K, batch, lr, B, s, bits = shape
+    out = {"loss_unquantised_average": loss(u.mean(0)), "loss_quantised": loss(param)}
+    if not (rank == 0 and world == 1 and not args.no_cpu):
+        return out
+    from oracle import qesgd_ref as ref
+    h_u = u.cpu().numpy()
+    t0 = time.perf_counter()
+    w0 = np.zeros(d, dtype=np.float32)
+    r_u = np.stack([ref.lr_local_epoch(X[k * n_local:(k + 1) * n_local], y[k * n_local:(k + 1) * n_local],
+                                       batch, lr, w0) for k in range(K)])
+    t_epoch = time.perf_counter() - t0
+    err = np.linalg.norm(h_u.astype(np.float64) - r_u, axis=1) / np.linalg.norm(r_u, axis=1)
+    t0 = time.perf_counter()
+    enc = [ref.encode(h_u[k], w0, B, s, bits, ref.SCALE_NORM, 0, k, 0) for k in range(K)]
+    r_codes, r_scales = np.stack([e[0] for e in enc]), np.stack([e[1] for e in enc])
+    r_param = ref.decode_average_apply(w0, r_codes, r_scales, B, s, bits)
+    t_codec = time.perf_counter() - t0
+    g_codes = codes.cpu().numpy().view(np.uint32).reshape(K, -1)[:, :r_codes.shape[1]]
+    g_scales = scales.cpu().numpy()[:, :r_scales.shape[1]]
+    g_param = param.cpu().numpy()
+    tol = 1e-6 * np.maximum(np.abs(r_param), np.repeat(r_scales.max(0), B)[:d])
+    out["oracle"] = {"local_epoch_rel_l2_err_max": float(err.max()), "local_epoch_within_1e-5": bool(err.max() <= 1e-5),
+                     "codes_bit_exact": bool((g_codes == r_codes).all()),
+                     "scales_bit_exact": bool((g_scales.view(np.uint32) == r_scales.view(np.uint32)).all()),
+                     "param_within_1e-6": bool((np.abs(g_param.astype(np.float64) - r_param) <= tol).all()),
+                     "oracle_local_epoch_s": t_epoch, "oracle_codec_s": t_codec, "cores": 1}
+    return out
 
 
 # ---------------------------------------------------------------- reference ---
