@@ -180,7 +180,8 @@ int qesgd_lr_sgd_step(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32_t
                       float lr, float *u);
 /* The summand of Eq. 2 alone: g_out = (1/m) * sum_j grad f_j(w) on the m rows of Xb, for
  * workers that push (quantised) gradients instead of parameters.  w and g_out are float[d]
- * and must not overlap.  Same two passes and accuracy as qesgd_lr_sgd_step. */
+ * and must not overlap.  One margin pass and one pass that writes the gradient; fp32
+ * arithmetic and accumulation as for qesgd_lr_sgd_step. */
 int qesgd_lr_gradient(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32_t m, uint64_t d,
                       const float *w, float *g_out);
 /* Rows [0, n_local) of X in consecutive minibatches of `batch` rows, in row
@@ -210,7 +211,9 @@ int qesgd_lr_local_epoch_batch(qesgd_ctx *ctx, const float *X, const float *y, u
  * inside a memory-pool or allocator callback, a real-time loop that must not touch
  * the driver's allocator, or a host that was handed a fixed memory budget and may
  * not create a qesgd_ctx (qesgd_create allocates).  It is qesgd_lr_sgd_step without
- * a context: same kernels, same arithmetic, same result.
+ * a context, always in the two-pass form (one margin pass, one update pass).  The context
+ * entry point may run the step in its persistent kernel instead, whose sums run in another
+ * order: the two agree to rounding (1e-5 relative), not bit for bit.
  *
  * The partial margins the two passes exchange live in a fixed array inside the
  * library image (64 KB of device memory on every GPU that loads the library, held
