@@ -121,7 +121,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const 
     }
 }
 // One 2-D box of the row-major matrix X: columns [x, x + box width), rows [y, y + SUB).
-// x * 4 bytes is a multiple of 16; dst is 128-byte aligned.  No multicast.
+// x * 4 bytes is a multiple of 16; dst is 128-byte aligned.  The copy goes to this CTA alone.
 __device__ __forceinline__ void tma_load_box(float *dst, const CUtensorMap *map, uint32_t x, uint32_t y,
                                              uint64_t *bar)
 {
