@@ -333,8 +333,12 @@ def load_traffic(kernel, workload):
     """DRAM bytes (read + write) per launch from the committed ncu summary; None when there is
     no capture for this kernel and workload, or the kernel source has changed since."""
     import hashlib
-    path = os.path.join(ROOT, "profiles", "dram_traffic_bench_c4.txt")
-    src = os.path.join(ROOT, "paper_1901_03040_b200", "csrc", "qesgd_codec.cu")
+    if kernel == "local_epoch":
+        path = os.path.join(ROOT, "profiles", "dram_traffic_bench_c1.txt")
+        src = os.path.join(ROOT, "paper_1901_03040_b200", "csrc", "qesgd_lr_epoch.cu")
+    else:
+        path = os.path.join(ROOT, "profiles", "dram_traffic_bench_c4.txt")
+        src = os.path.join(ROOT, "paper_1901_03040_b200", "csrc", "qesgd_codec.cu")
     try:
         with open(src, "rb") as fh:
             sha = hashlib.sha256(fh.read()).hexdigest()
@@ -600,7 +604,7 @@ def run_c1(args, device, world, rank):
                          "achieved": n * d * 4 / (statistics.mean(times["local_epoch"]) * 1e-3) / 1e9,
                          "peak": peaks()[0], "unit": "GB/s",
                          "frac": n * d * 4 / (statistics.mean(times["local_epoch"]) * 1e-3) / 1e9 / peaks()[0],
-                         "traffic": None, "peak_source": peaks()[1],
+                         "traffic": load_traffic("local_epoch", "c1"), "peak_source": peaks()[1],
                          "algorithmic_bytes_per_launch": float(n * d * 4)},
             "status_flags": ctx.qesgd_status(),
             "x_bytes_per_epoch": int(n * d * 4),
