@@ -594,6 +594,11 @@ int qesgd_launch_lr_epoch_fused(const float *X, const float *y, uint64_t n_local
     void *params[] = {(void *)&a, (void *)&map_a, (void *)&map_b};
     e = cudaLaunchCooperativeKernel((const void *)qesgd_lr_epoch_kernel, dim3(ncta), dim3(EP_THREADS), params,
                                     smem, stream);
+    if (e == cudaErrorCooperativeLaunchTooLarge || e == cudaErrorLaunchOutOfResources ||
+        e == cudaErrorInvalidConfiguration || e == cudaErrorNotSupported) {
+        cudaGetLastError();   // the device cannot hold all CTAs at once as configured: two-pass steps
+        return -1;
+    }
     if (e != cudaSuccess) return (int)e;
     *launched = 1;
     return 0;
