@@ -17,7 +17,14 @@
 //         then fence + one atomic increment of counter[i]
 //   W(i)  wait until counter[i] == number of CTAs, sum the partials of every row in a
 //         fixed order, coefficients (lr/m) y_j / (1 + exp(y_j m_j)) into shared memory
-//   U(i)  u[cols] += sum_j coef_j x_j from the buffer, then the buffer is released
+//   U(i)  u[cols] += sum_j coef_j x_j from the tile
+//
+// Where the minibatch has at most 64 rows the tile does not wait in shared memory between M
+// and U: right after M every thread moves its share of it into tensor memory (tcgen05.st;
+// the SM's 256 KB of it hold one tile per consumer group and are otherwise unused here) and
+// the shared-memory slots go back to the producer, so the next tile's copies run while this
+// one waits for the other CTAs; U reads the tile back with tcgen05.ld.  Larger minibatches
+// stay in shared memory and release their slots during U.
 //
 // Each tile's M, W, U is a chain of dependent round trips to global memory (fence, count,
 // partial margins) that lasts longer than the tile's own transfer from HBM.  The eight
@@ -138,6 +145,49 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p)
     return v;
 }
 
+// ---- tensor memory as a stash for a tile between its two uses --------------------------
+// The SM's 256 KB of tensor memory (128 lanes x 512 columns of 32 bits) is not needed for
+// any matrix product here, so it holds a consumer group's tile while the group waits for the
+// other CTAs: thread t of a warp owns lane 32 * (warp % 4) + t and reads back exactly what it
+// stored, so no ordering between threads is involved.  One access moves 32 registers of
+// every thread of the warp (the 8 rows x 4 columns a thread takes of a sub-tile).
+__device__ __forceinline__ void tmem_alloc_all(uint32_t *smem_result)   // one whole warp
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(smem_result))
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_free_all(uint32_t taddr)           // the same warp
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float4 (&v)[8])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, "
+        "%14, %15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "f"(v[0].x), "f"(v[0].y), "f"(v[0].z), "f"(v[0].w), "f"(v[1].x), "f"(v[1].y), "f"(v[1].z), "f"(v[1].w),
+        "f"(v[2].x), "f"(v[2].y), "f"(v[2].z), "f"(v[2].w), "f"(v[3].x), "f"(v[3].y), "f"(v[3].z), "f"(v[3].w),
+        "f"(v[4].x), "f"(v[4].y), "f"(v[4].z), "f"(v[4].w), "f"(v[5].x), "f"(v[5].y), "f"(v[5].z), "f"(v[5].w),
+        "f"(v[6].x), "f"(v[6].y), "f"(v[6].z), "f"(v[6].w), "f"(v[7].x), "f"(v[7].y), "f"(v[7].z), "f"(v[7].w)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float4 (&v)[8])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, "
+        "%15, %16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=f"(v[0].x), "=f"(v[0].y), "=f"(v[0].z), "=f"(v[0].w), "=f"(v[1].x), "=f"(v[1].y), "=f"(v[1].z),
+          "=f"(v[1].w), "=f"(v[2].x), "=f"(v[2].y), "=f"(v[2].z), "=f"(v[2].w), "=f"(v[3].x), "=f"(v[3].y),
+          "=f"(v[3].z), "=f"(v[3].w), "=f"(v[4].x), "=f"(v[4].y), "=f"(v[4].z), "=f"(v[4].w), "=f"(v[5].x),
+          "=f"(v[5].y), "=f"(v[5].z), "=f"(v[5].w), "=f"(v[6].x), "=f"(v[6].y), "=f"(v[6].z), "=f"(v[6].w),
+          "=f"(v[7].x), "=f"(v[7].y), "=f"(v[7].z), "=f"(v[7].w)
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
 // Sum over the 32 lanes of 8 per-lane values at once: three halving exchanges leave one
 // value per lane, two plain butterflies finish.  Lane L ends with the total of value
 // 4*bit4(L) + 2*bit3(L) + bit2(L); the order of the additions is fixed.
@@ -207,10 +257,18 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
     if (tid == 0) {
         for (uint32_t s = 0; s < 2u * a.nsub_max; ++s) mbar_init(&full[s], 1u);
         for (uint32_t s = 0; s < 2u * a.nsub_max; ++s) mbar_init(&consumed[s], EP_GROUP / 32);
-        for (int f = 0; f < 8; ++f) s_flag[f] = 0u;
+        for (int f = 0; f < 16; ++f) s_flag[f] = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    // Minibatches of at most 64 rows (8 sub-tiles x 32 registers x 2 groups = all 512 columns)
+    // are stashed in tensor memory between their two uses; larger ones stay in shared memory.
+    const bool stash = a.nsub_max <= 8u;
+    if (stash && warp == 0) tmem_alloc_all(const_cast<uint32_t *>(&s_flag[8]));
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_base = s_flag[8];
 
     // ------------------------------------------------------------ producer ----
     if (warp == EP_CONSUMERS / 32) {
@@ -274,6 +332,14 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
     const bool early_u = (a.K & 1u) == 0u && a.K >= 4u;
     float4 un[EP_MAX_COLS / 128];
     if (early_u && g < ntiles) load_u(g % a.K, un);
+
+    // the update's (and the stash's) share of a tile: four columns, all rows
+    const uint32_t col = tg * 4u;
+    const bool colok = col < a.cols && (uint64_t)c0 + col < a.d;
+    const bool first = col < (uint32_t)EP_BOX_COLS;
+    const uint32_t off = first ? col : SUB * cols_a + (col - EP_BOX_COLS);
+    const uint32_t pitch = first ? cols_a : cols_b;
+    const uint32_t taddr = tmem_base + ((32u * wg) << 16) + 256u * g;   // this thread's lane, this group's columns
 
     for (uint32_t i = g; i < ntiles; i += 2u) {
         const Tile T = tile_of(a, i);
@@ -348,6 +414,26 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
             }
         }
 
+        // ---- stash: the tile moves from shared to tensor memory and its slots go back to the
+        // producer now, so that the copies of the group's next tile run during the exchange ----
+        if (stash) {
+            // every warp observes the arrival of every sub-tile itself (lane s looks at sub-tile s)
+            for (uint32_t s = lane; s < T.nsub; s += 32u) mbar_wait(&bars[s], parity, &s_flag[0]);
+            __syncwarp();
+            for (uint32_t s = 0; s < T.nsub; ++s) {
+                const float *__restrict__ base = buf + (size_t)s * slot_floats + off;
+                float4 x[SUB];
+#pragma unroll
+                for (uint32_t r = 0; r < (uint32_t)SUB; ++r)
+                    x[r] = colok ? *reinterpret_cast<const float4 *>(base + (size_t)r * pitch)
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+                tmem_st32(taddr + 32u * s, x);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&consumed[g * a.nsub_max + s]);
+            }
+            tmem_wait_st();
+        }
+
         // ---- W(i): all CTAs' partial margins -> step coefficients in shared memory ----
         {
             // the labels of the rows this lane will finish, requested before the wait
@@ -407,11 +493,6 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
 
         // ---- U(i): update this CTA's columns of u from the buffer, release the buffer ----
         {
-            const uint32_t col = tg * 4u;
-            const bool colok = col < a.cols && (uint64_t)c0 + col < a.d;
-            const bool first = col < (uint32_t)EP_BOX_COLS;
-            const uint32_t off = first ? col : SUB * cols_a + (col - EP_BOX_COLS);
-            const uint32_t pitch = first ? cols_a : cols_b;
             float4 *const up = reinterpret_cast<float4 *>(a.u + (uint64_t)T.k * a.u_stride + c0 + col);
             float4 uold = make_float4(0.f, 0.f, 0.f, 0.f);
             if (colok) uold = *up;                       // requested now, needed after the loop
@@ -419,10 +500,27 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
             // wrote: lane s looks at sub-tile s (a look costs about 0.1 us, so the lanes look in
             // parallel), and the warp follows its lanes through __syncwarp.  All of them have
             // landed: the warps that took the margins waited for them.
-            for (uint32_t s = lane; s < T.nsub; s += 32u) mbar_wait(&bars[s], parity, &s_flag[0]);
+            if (!stash)
+                for (uint32_t s = lane; s < T.nsub; s += 32u) mbar_wait(&bars[s], parity, &s_flag[0]);
             __syncwarp();
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (uint32_t s = 0; s < T.nsub; ++s) {
+            for (uint32_t s = 0; stash && s < T.nsub; ++s) {
+                float4 x[SUB];
+                tmem_ld32(taddr + 32u * s, x);
+                tmem_wait_ld();
+#pragma unroll
+                for (uint32_t r = 0; r < (uint32_t)SUB; ++r) {
+                    const uint32_t jj = s * SUB + r;
+                    if (colok && jj < T.m) {
+                        const float cj = coef[jj];
+                        acc.x = fmaf(cj, x[r].x, acc.x);
+                        acc.y = fmaf(cj, x[r].y, acc.y);
+                        acc.z = fmaf(cj, x[r].z, acc.z);
+                        acc.w = fmaf(cj, x[r].w, acc.w);
+                    }
+                }
+            }
+            for (uint32_t s = 0; !stash && s < T.nsub; ++s) {
                 if (colok) {
                     const float *__restrict__ base = buf + (size_t)s * slot_floats + off;
 #pragma unroll
@@ -460,6 +558,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
 
     // Both groups meet here, whether they finished or gave up.
     asm volatile("bar.sync 3, %0;" ::"n"(EP_CONSUMERS) : "memory");
+    if (stash && warp == 0) tmem_free_all(tmem_base);   // on every path out of the kernel
     if (s_flag[0] == 0u) return;
 
     // ---- a wait ran out: tell the others, let the copies in flight land, leave --------
@@ -570,7 +669,7 @@ int qesgd_launch_lr_epoch_fused(const float *X, const float *y, uint64_t n_local
 
     // shared memory: two tile buffers | coefficients of both groups | barriers | flags
     const size_t smem = (size_t)2 * a.nsub_max * SUB * cols * sizeof(float) + 2 * EP_MAX_M * sizeof(float) +
-                        (4 * EP_MAX_NSUB) * sizeof(uint64_t) + 32;
+                        (4 * EP_MAX_NSUB) * sizeof(uint64_t) + 64;
     if (smem > (size_t)limit) return -1;
 
     // workspace: header | one counter per tile | partial margins
