@@ -145,6 +145,26 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p)
     return v;
 }
 
+// Barrier `id` of `count` threads that also answers one question the same way for all of them:
+// has any of them seen `flag` set?  (Each thread reads the flag for itself; a plain barrier
+// followed by separate reads could send the threads different ways while another warp sets it,
+// and the ones that stay would then wait at the next barrier for the ones that left.)
+__device__ __forceinline__ bool sync_any(uint32_t id, uint32_t count, uint32_t flag)
+{
+    uint32_t r;
+    asm volatile(
+        "{\n"
+        ".reg .pred p, q;\n"
+        "setp.ne.u32 q, %1, 0;\n"
+        "bar.red.or.pred p, %2, %3, q;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}"
+        : "=r"(r)
+        : "r"(flag), "r"(id), "r"(count)
+        : "memory");
+    return r != 0u;
+}
+
 // ---- tensor memory as a stash for a tile between its two uses --------------------------
 // The SM's 256 KB of tensor memory (128 lanes x 512 columns of 32 bits) is not needed for
 // any matrix product here, so it holds a consumer group's tile while the group waits for the
@@ -361,8 +381,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
                 }
                 __threadfence_block();
             }
-            group_sync();
-            if (s_flag[0] != 0u) break;
+            if (sync_any(1u + g, EP_GROUP, s_flag[0])) break;
         }
 
         // ---- M(i): margins over this CTA's columns, then the signal to the other CTAs ----
@@ -406,8 +425,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
                 if ((lane & 3u) == 0u && jj < T.m) pout[(uint64_t)jj * a.gpad] = tot;
             }
             if (!ok) s_flag[0] = 1u;
-            group_sync();
-            if (s_flag[0] != 0u) break;
+            if (sync_any(1u + g, EP_GROUP, s_flag[0])) break;
             if (tg == 0) {
                 asm volatile("fence.acq_rel.gpu;" ::: "memory");   // partials before the count
                 atomicAdd(a.counters + i, 1u);
@@ -451,8 +469,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
                     }
                 }
             }
-            group_sync();
-            if (s_flag[0] != 0u) break;
+            if (sync_any(1u + g, EP_GROUP, s_flag[0])) break;
             // a warp sums eight rows at a time: lanes along the CTA index (contiguous in memory)
             const float *__restrict__ pin = a.partial + ((uint64_t)(i % EP_RING) * a.batch) * a.gpad;
             // Two passes of eight rows per iteration; all 32 loads of a lane are requested
