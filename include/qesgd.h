@@ -72,8 +72,8 @@ extern "C" {
 typedef struct qesgd_ctx qesgd_ctx;
 
 /* Create a context bound to `device` and to `cuda_stream` (a cudaStream_t passed
- * as void*; NULL = the legacy default stream).  Allocates a few KB of device
- * memory (status word, logistic-regression workspace) that qesgd_destroy frees.
+ * as void*; NULL = the legacy default stream).  Allocates 256 bytes (status word) and
+ * 4 MiB (logistic-regression workspace) of device memory that qesgd_destroy frees.
  * This is the only call that allocates. */
 int qesgd_create(qesgd_ctx **out, int device, void *cuda_stream);
 int qesgd_destroy(qesgd_ctx *ctx);
@@ -151,7 +151,7 @@ int qesgd_requantize(qesgd_ctx *ctx, float *u, const float *anchor, uint64_t d, 
                      uint32_t *codes_out, float *scales_out);
 
 /*
- * Gradient compression on the push side (Sec. 3: "users can compress gradients"; the QSGD
+ * Gradient compression on the push side (Sec. 3, remark after Algorithm 3; the QSGD
  * baseline of Sec. 5 quantises gradients with delta = ||g||): the K streams hold quantised
  * gradients, encoded with anchor == NULL, and the server takes
  *   param_i <- param_i + alpha * (1/K) * sum_k (+-level_{k,i} * fl32(scale_{k,bucket(i)} / s))
@@ -222,9 +222,12 @@ int qesgd_lr_local_epoch_batch(qesgd_ctx *ctx, const float *X, const float *y, u
  *     QESGD_ELIMIT and enqueue nothing.  d is unlimited.
  *   - the call works on the CURRENT device and enqueues on cuda_stream (NULL = legacy
  *     default stream); Xb, yb, u are device pointers as for qesgd_lr_sgd_step.
- *   - it calls no cudaMalloc / cudaFree and nothing that allocates.  The first call
- *     on each device looks up the array's device address (a query, not an
- *     allocation); make that first call before starting any stream capture.
+ *   - it calls no cudaMalloc / cudaFree and no allocating library routine.  The first
+ *     call on each device looks up the array's device address; with lazy module loading
+ *     that query may be the moment the driver loads this library's device image (and
+ *     places the array).  So make one warm-up call per device OUTSIDE the region in which
+ *     allocation is forbidden, and before starting any stream capture; later calls only
+ *     launch two kernels.
  *   - every call shares the one array, which keeps the previous call's contents.
  *     Nothing in it has to start at zero: the first pass overwrites every slot the
  *     second pass reads.  Two calls that overlap on the GPU (different streams, or

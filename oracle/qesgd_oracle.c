@@ -322,7 +322,7 @@ int qesgd_ref_requantize(float *u, const float *anchor, uint64_t n, uint64_t i0,
     return QREF_OK;
 }
 
-/* Gradient compression on the push side (Sec. 3: "users can compress gradients"; the QSGD
+/* Gradient compression on the push side (Sec. 3, remark after Algorithm 3; the QSGD
  * baseline of Sec. 5 quantises gradients): the K streams hold quantised gradients and the
  * server takes w <- w + alpha * (1/K) sum_k g_k with alpha = -learning rate (Eq. 2 with the
  * minibatch mean replaced by the mean of the decoded workers).  alpha = 1 is the averaging

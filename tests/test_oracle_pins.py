@@ -323,9 +323,10 @@ def test_brute_force_expectation_small_d(mode, s, bits):
         r_fp = np.float32(abs(z[i])) * inv
         assert set(np.unique(lv)) <= {math.floor(r_fp), math.floor(r_fp) + 1}
         # ... and its mean level is the exact r = |z| / delta up to 2^-17 from the draw
-        # resolution and two fp32 roundings (inv and the product), each <= r * 2^-24
+        # resolution and two fp32 roundings (inv and the product), each a factor within
+        # 1 +- 2^-24: |r_fp - r| <= r * ((1 + 2^-24)^2 - 1) = r * (2^-23 + 2^-48)
         mean_level = F(int(lv.sum()), 65536)
-        assert abs(mean_level - (lo + p)) <= F(1, 131072) + (lo + 1) * F(1, 1 << 22)
+        assert abs(mean_level - (lo + p)) <= F(1, 131072) + (lo + p) * (F(1, 1 << 23) + F(1, 1 << 48))
         floors.append(lo)
         probs.append(p)
     mean = [F(0)] * d
@@ -461,6 +462,51 @@ def test_fixed_delta_clips_at_the_top_level():
         assert lv[4] in (-2, -3)
         ups += lv[4] == -3
     assert 60 < ups < 140        # p = 1/2
+
+
+def test_fixed_delta_nonfinite_values_are_handled_element_by_element():
+    """Caller-given spacing, non-finite input (first and last branch of Eq. 4 read on the
+    extended reals): +Inf lies above the range and takes the top grid point +s, -Inf the
+    bottom one -s, for every draw; NaN is no point of the line at all: code 0 and the
+    NONFINITE status.  Nothing couples the elements of a bucket in this mode, so the finite
+    neighbours must come out exactly as they do when the non-finite values are replaced by
+    zeros, draw for draw."""
+    s, bits, delta, B = 7, 4, np.float32(2.0 ** -8), 64
+    rng = np.random.default_rng(11)
+    base = (rng.standard_normal(2 * B) * 3 * delta).astype(np.float32)
+    base[5], base[B + 9] = 2.5 * delta, -6.25 * delta          # known neighbours
+    pos, neg, nan = [3, B + 1], [17, B + 40], [30, B + 63]
+    bad = base.copy()
+    bad[pos], bad[neg], bad[nan] = np.inf, -np.inf, np.nan
+    clean = base.copy()
+    clean[pos + neg + nan] = 0.0
+    seen_5, seen_9 = set(), set()
+    for epoch in range(64):
+        codes, scales, status = q.encode(bad, None, B, s, bits, q.SCALE_FIXED, 9, 2, epoch,
+                                         fixed_delta=float(delta))
+        ref_codes, ref_scales, ref_status = q.encode(clean, None, B, s, bits, q.SCALE_FIXED, 9, 2,
+                                                     epoch, fixed_delta=float(delta))
+        assert status == q.STATUS_NONFINITE and ref_status == 0
+        assert (scales == np.float32(s) * delta).all() and (ref_scales == scales).all()
+        raw = _unpack(codes, 2 * B, bits)
+        lv, ref_lv = _signed_levels(codes, 2 * B, bits), _signed_levels(ref_codes, 2 * B, bits)
+        assert (lv[pos] == s).all() and (raw[pos] == s).all()              # +Inf -> +s
+        assert (lv[neg] == -s).all() and (raw[neg] == (8 | s)).all()       # -Inf -> -s, sign bit set
+        assert (raw[nan] == 0).all()                                       # NaN -> code 0
+        others = np.setdiff1d(np.arange(2 * B), pos + neg + nan)
+        assert (lv[others] == ref_lv[others]).all()                        # neighbours untouched
+        assert lv[5] in (2, 3) and lv[B + 9] in (-6, -7)
+        seen_5.add(int(lv[5]))
+        seen_9.add(int(lv[B + 9]))
+    assert seen_5 == {2, 3} and seen_9 == {-6, -7}     # the neighbours' draws are alive
+    # a bucket with only NaN flags, a bucket with only +-Inf does not
+    only_inf = np.zeros(B, dtype=np.float32)
+    only_inf[0], only_inf[1] = np.inf, -np.inf
+    codes, _, status = q.encode(only_inf, None, B, s, bits, q.SCALE_FIXED, 1, 0, 0, fixed_delta=float(delta))
+    assert status == 0 and list(_signed_levels(codes, B, bits)[:3]) == [s, -s, 0]
+    # decode gives +-s*delta back for the clipped infinities
+    out = q.decode(codes, np.full(1, np.float32(s) * delta, dtype=np.float32), B, B, s, bits)
+    assert out[0] == s * delta and out[1] == -s * delta and not out[2:].any()
 
 
 # --------------------------------------------- logistic regression, Eq. 2 ----

@@ -24,8 +24,13 @@ def _step_noalloc(X, y, m, d, lr, u):
     assert rc == qesgd.OK, qesgd.lib.qesgd_strerror(rc)
 
 
-@pytest.mark.parametrize("m,d", [(64, 65536), (100, 3001), (256, 4096)])
-def test_noalloc_step_matches_the_context_entry_point_twice_in_a_row(m, d):
+@pytest.mark.parametrize("m,d", [(64, 65536), (100, 3001), (256, 4096), (256, 65536)])
+def test_noalloc_step_matches_the_oracle_and_the_context_entry_point_twice_in_a_row(m, d):
+    """Two calls in a row, the second continuing from the first one's result.  Each result is
+    compared with the fp64 CPU oracle's step from the same starting point (the tolerance of
+    the logistic step, 1e-5) and then with what the context entry point gives.  The last shape
+    (256 rows, 64 column segments) uses every float of the fixed array."""
+    from oracle import qesgd_ref as ref
     torch.cuda.set_device(0)
     X, y, _ = synthetic.logistic_problem(2 * m, d, seed=m + d)
     tX, ty = torch.from_numpy(X).cuda(), torch.from_numpy(y).cuda()
@@ -33,13 +38,20 @@ def test_noalloc_step_matches_the_context_entry_point_twice_in_a_row(m, d):
     want = torch.from_numpy(u0).cuda()
     got = torch.from_numpy(u0).cuda()
     ctx = qesgd.Context(0, None)
-    for call in range(2):                 # the second call continues from the first one's result
+    for call in range(2):
         rows = slice(call * m, (call + 1) * m)
         xb, yb = tX[rows].contiguous(), ty[rows].contiguous()
+        start = got.cpu().numpy()
+        oracle = ref.lr_sgd_step(X[rows], y[rows], 0.1, start).astype(np.float64)
         ctx.qesgd_lr_sgd_step(xb, yb, m, d, 0.1, want)
         _step_noalloc(xb, yb, m, d, 0.1, got)
         torch.cuda.synchronize()
         w, g = want.cpu().numpy().astype(np.float64), got.cpu().numpy().astype(np.float64)
+        assert np.linalg.norm(g - oracle) <= 1e-5 * np.linalg.norm(oracle)
+        assert np.abs(g - oracle).max() <= 1e-5 * np.abs(oracle).max()
+        # the step itself (not only the vector it is added to) is right
+        step_ref = oracle - start.astype(np.float64)
+        assert np.linalg.norm((g - start) - step_ref) <= 1e-3 * np.linalg.norm(step_ref)
         assert np.linalg.norm(g - w) <= 1e-5 * np.linalg.norm(w)
         assert np.abs(g - w).max() <= 1e-5 * np.abs(w).max()
         assert not np.array_equal(g, u0)
