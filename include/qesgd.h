@@ -195,15 +195,32 @@ int qesgd_lr_local_epoch(qesgd_ctx *ctx, const float *X, const float *y, uint64_
  * of all K workers is ONE persistent kernel, launched cooperatively with one CTA per SM,
  * that stages every minibatch in shared memory by TMA and reads X from HBM once; its
  * CTAs exchange partial margins through the context's workspace, which the call clears
- * first.  Every wait inside it is bounded (about a second): should one run out, the
- * kernel returns, u is left partly updated and QESGD_STATUS_TIMEOUT is set in the status
- * word.  The kernel needs all its CTAs resident at once, so do not run it next to other
- * kernels that occupy the device for long.  Other shapes run one margin pass and one
+ * first.  Every wait the kernel loops on (for another CTA, another warp group, a copy) is
+ * bounded by the context's wait limit (one second unless qesgd_set_wait_limit changed it):
+ * should one run out, the kernel returns, u is left partly updated and
+ * QESGD_STATUS_TIMEOUT is set in the status word; the context stays usable and the next call
+ * starts clean.  One wait has no bound of its own: at its start the kernel allocates the
+ * SM's tensor memory, and that allocation blocks while another kernel resident on the same
+ * SM (another stream or process) holds tensor memory, until that kernel ends.  The kernel
+ * needs all its CTAs resident at once, so do not run it next to other kernels that occupy
+ * the device for long.  Other shapes run one margin pass and one
  * update pass per minibatch, step t of every worker in the same launches.  Results are
  * deterministic (fixed summation order) on either path. */
 int qesgd_lr_local_epoch_batch(qesgd_ctx *ctx, const float *X, const float *y, uint64_t n_local,
                                uint64_t d, uint32_t K, uint32_t batch, float lr, float *u,
                                uint64_t u_stride);
+
+/* Limit, in nanoseconds, of each wait inside the persistent local-epoch kernel (its CTAs
+ * wait for one another's partial margins and for their own TMA copies).  0 restores the
+ * default of one second; at most 10 seconds.  A limit below one microsecond means "look once
+ * more, then give up" (the device timer is not finer than that).  Takes effect with the next
+ * qesgd_lr_local_epoch[_batch] / qesgd_lr_sgd_step call of this context. */
+int qesgd_set_wait_limit(qesgd_ctx *ctx, uint64_t nanoseconds);
+/* Test hook for the give-up path of that kernel (no counterpart in the paper): CTA number
+ * `cta` does not announce its partial margins of the first minibatch, so every CTA's wait
+ * for them runs out after the wait limit, the kernel returns and QESGD_STATUS_TIMEOUT is
+ * set.  Nothing faults or hangs.  cta = -1 (the default) switches the hook off. */
+int qesgd_debug_drop_signal(qesgd_ctx *ctx, int64_t cta);
 
 /*
  * The paper has no counterpart for this entry point; it exists for callers that are

@@ -69,6 +69,8 @@ int qesgd_create(qesgd_ctx **out, int device, void *cuda_stream)
     ctx->d_status = nullptr;
     ctx->d_lr_work = nullptr;
     ctx->lr_work_floats = QESGD_LR_WORK_FLOATS;
+    ctx->wait_ns = QESGD_DEFAULT_WAIT_NS;
+    ctx->drop_cta = 0xFFFFFFFFu;
     DeviceGuard guard(device);
     if (!guard.ok) { delete ctx; return QESGD_ECUDA; }
     cudaError_t e = cudaMalloc((void **)&ctx->d_status, 256);
@@ -103,6 +105,20 @@ int qesgd_set_stream(qesgd_ctx *ctx, void *cuda_stream)
 {
     if (!ctx) return QESGD_EINVAL;
     ctx->stream = (cudaStream_t)cuda_stream;
+    return QESGD_OK;
+}
+
+int qesgd_set_wait_limit(qesgd_ctx *ctx, uint64_t nanoseconds)
+{
+    if (!ctx || nanoseconds > QESGD_MAX_WAIT_NS) return QESGD_EINVAL;
+    ctx->wait_ns = nanoseconds == 0 ? QESGD_DEFAULT_WAIT_NS : nanoseconds;
+    return QESGD_OK;
+}
+
+int qesgd_debug_drop_signal(qesgd_ctx *ctx, int64_t cta)
+{
+    if (!ctx || cta < -1 || cta > 0x7FFFFFFF) return QESGD_EINVAL;
+    ctx->drop_cta = cta < 0 ? 0xFFFFFFFFu : (uint32_t)cta;
     return QESGD_OK;
 }
 
@@ -296,7 +312,8 @@ int qesgd_lr_local_epoch_batch(qesgd_ctx *ctx, const float *X, const float *y, u
         int launched = 0;
         const int e = qesgd_launch_lr_epoch_fused(X, y, n_local, d, K, batch, lr, u, K > 1 ? u_stride : 0,
                                                   ctx->d_lr_work, ctx->lr_work_floats, ctx->d_status,
-                                                  ctx->device, ctx->sm_count, ctx->stream, &launched);
+                                                  ctx->device, ctx->sm_count, ctx->wait_ns, ctx->drop_cta,
+                                                  ctx->stream, &launched);
         ctx->launches += (uint64_t)launched;
         if (e > 0) return cuda_fail(ctx, e);
         if (e == 0) return QESGD_OK;

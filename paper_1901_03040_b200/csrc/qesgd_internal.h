@@ -16,7 +16,11 @@ struct qesgd_ctx {
     uint64_t launches;
     int last_cuda_error;
     int sm_count;
+    uint64_t wait_ns;       // limit of each wait inside the local-epoch kernel
+    uint32_t drop_cta;      // give-up-path test hook of the local-epoch kernel (none: ~0)
 };
+static const uint64_t QESGD_DEFAULT_WAIT_NS = 1000000000ull;
+static const uint64_t QESGD_MAX_WAIT_NS = 10000000000ull;
 
 // Workspace for partial margins: K * P * m floats must fit.
 static const uint64_t QESGD_LR_WORK_FLOATS = 1ull << 20;
@@ -110,4 +114,5 @@ int qesgd_launch_lr_gradient(const float *Xb, const float *yb, uint32_t m, uint6
 int qesgd_launch_lr_epoch_fused(const float *X, const float *y, uint64_t n_local, uint64_t d,
                                 uint32_t K, uint32_t batch, float lr, float *u, uint64_t u_stride,
                                 float *work, uint64_t work_floats, uint32_t *status, int device,
-                                int sm_count, cudaStream_t stream, int *launched);
+                                int sm_count, uint64_t wait_ns, uint32_t drop_cta, cudaStream_t stream,
+                                int *launched);

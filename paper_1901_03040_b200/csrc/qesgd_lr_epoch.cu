@@ -35,9 +35,14 @@
 // odd K a group waits for the other group's update before it takes the margins.
 //
 // The CTAs wait on one another, so the kernel is launched cooperatively (all CTAs are
-// resident by construction: at most one per SM).  Every wait is bounded: a wait that
-// runs out sets QESGD_STATUS_TIMEOUT and an abort word that the other CTAs poll; each CTA
-// then waits (bounded again) for its own copies in flight and returns.
+// resident by construction: at most one per SM).  Every wait the kernel itself loops on is
+// bounded by the context's wait limit: a wait that runs out sets QESGD_STATUS_TIMEOUT and an
+// abort word that the other CTAs poll, and the CTA's consumer warps leave.  The producer warp
+// is the last to go on every path: it waits (on a bound of its own) for each copy it has
+// requested and nobody has consumed, so no CTA ends with a copy still writing its shared
+// memory.  The one wait without a bound is the tensor-memory allocation at the start, which
+// blocks while another kernel resident on the same SM holds tensor memory (until that kernel
+// ends).
 #include <cuda.h>
 
 #include <mutex>
@@ -55,7 +60,8 @@ constexpr int EP_MAX_COLS = 512;     // columns per CTA: 128 groups of 4
 constexpr int EP_BOX_COLS = 256;     // widest TMA box
 constexpr int EP_MAX_M = 256;        // rows per minibatch the fused path takes
 constexpr int EP_MAX_NSUB = EP_MAX_M / SUB;
-constexpr uint64_t WAIT_LIMIT_NS = 1000000000ull;   // one second per wait
+constexpr uint64_t DRAIN_LIMIT_NS = 2000000000ull;   // the producer's last wait for its own copies
+constexpr uint64_t COARSE_TIMER_NS = 1024ull;        // limits below this mean "one look, then give up"
 constexpr uint32_t EP_HEADER_WORDS = 64;             // word 0 = abort flag
 
 struct EpochArgs {
@@ -75,6 +81,9 @@ struct EpochArgs {
     uint32_t *counters;     // one per tile, zero at launch
     float *partial;         // [EP_RING][batch][gpad], columns >= gridDim.x stay zero
     uint32_t *status;
+    uint64_t wait_ns;       // limit of every wait on another CTA, warp group or copy
+    uint32_t poll_mask;     // the clock is read every (poll_mask + 1) looks at a counter
+    uint32_t drop_cta;      // test hook: this CTA does not count itself for tile 0 (none: ~0)
 };
 
 // ------------------------------------------------------------- primitives ----
@@ -116,15 +125,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity)
         : "memory");
     return ok != 0u;
 }
+// Has a wait that began at t0 used up `limit`?  The global timer may tick as coarsely as a
+// microsecond, so a smaller limit is read as "give up after one round of looks".
+__device__ __forceinline__ bool expired(uint64_t t0, uint64_t limit)
+{
+    return limit < COARSE_TIMER_NS || now_ns() - t0 > limit;
+}
 // Bounded wait for phase `parity` of a barrier; gives up early when `*stop` is set.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const volatile uint32_t *stop)
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, const volatile uint32_t *stop,
+                                          uint64_t limit)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const uint64_t t0 = now_ns();
     for (;;) {
         for (int n = 0; n < 32; ++n)
             if (mbar_try_wait(bar, parity)) return true;
-        if (*stop != 0u || now_ns() - t0 > WAIT_LIMIT_NS) return false;
+        if (*stop != 0u || expired(t0, limit)) return false;
     }
 }
 // One 2-D box of the row-major matrix X: columns [x, x + box width), rows [y, y + SUB).
@@ -264,8 +280,8 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
     float *const s_coef = tile + (size_t)2u * a.nsub_max * slot_floats;
     uint64_t *const full = reinterpret_cast<uint64_t *>(s_coef + 2 * EP_MAX_M);
     uint64_t *const consumed = full + 2 * EP_MAX_NSUB;
-    // [0] a wait ran out in this CTA, [1] tiles the producer has requested, [2] producer has
-    // stopped, [3] always zero, [4], [5] tiles completed by consumer group 0, 1
+    // [0] a wait ran out in this CTA, [3] always zero, [4], [5] tiles completed by consumer
+    // group 0, 1, [8] base address of the tensor memory
     volatile uint32_t *const s_flag = reinterpret_cast<volatile uint32_t *>(consumed + 2 * EP_MAX_NSUB);
 
     const uint32_t tid = threadIdx.x, lane = tid & 31u, warp = tid >> 5;
@@ -292,6 +308,9 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
 
     // ------------------------------------------------------------ producer ----
     if (warp == EP_CONSUMERS / 32) {
+        // Lane L remembers, for slots L and L + 32 of the 2 * nsub_max slots, the tile whose copy
+        // was requested into the slot last (none: ~0).
+        uint32_t last_tile[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};
         for (uint32_t i = 0; i < ntiles; ++i) {
             const uint32_t b = i & 1u;
             const Tile T = tile_of(a, i);
@@ -300,8 +319,13 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
             for (uint32_t s = 0; s < T.nsub && ok; ++s) {
                 // a slot is free once the update of tile i-2 has read sub-tile s
                 if (i >= 2u)
-                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(&consumed[b * a.nsub_max + s],
-                                                           ((i - 2u) >> 1) & 1u, &s_flag[0])) != 0;
+                    ok = __all_sync(0xFFFFFFFFu, mbar_wait(&consumed[b * a.nsub_max + s], ((i - 2u) >> 1) & 1u,
+                                                           &s_flag[0], a.wait_ns)) != 0;
+                if (ok) {
+                    const uint32_t q = b * a.nsub_max + s;
+                    if (q == lane) last_tile[0] = i;
+                    if (q == lane + 32u) last_tile[1] = i;
+                }
                 if (ok && lane == 0) {
                     uint64_t *const bar = &full[b * a.nsub_max + s];
                     float *const dst = tile + (size_t)(b * a.nsub_max + s) * slot_floats;
@@ -318,14 +342,16 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
                 }
                 break;
             }
-            __syncwarp();
-            if (lane == 0) s_flag[1] = i + 1u;
         }
+        // Last out, on every path: each slot's latest copy has been consumed (then it has
+        // landed) or is waited for here, so that the CTA does not end -- and its shared memory
+        // is not handed to another CTA -- while a copy is still writing it.  After a normal
+        // epoch these waits end with the consumers' last tiles.
         __syncwarp();
-        if (lane == 0) {
-            __threadfence_block();
-            s_flag[2] = 1u;
-        }
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+            if (last_tile[h] != 0xFFFFFFFFu)
+                mbar_wait(&full[lane + 32u * h], (last_tile[h] >> 1) & 1u, &s_flag[3], DRAIN_LIMIT_NS);
         return;
     }
 
@@ -374,7 +400,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
             if (tg == 0) {
                 const uint64_t t0 = now_ns();
                 while (s_flag[4u + (g ^ 1u)] < need) {
-                    if (s_flag[0] != 0u || now_ns() - t0 > WAIT_LIMIT_NS) {
+                    if (s_flag[0] != 0u || expired(t0, a.wait_ns)) {
                         s_flag[0] = 1u;
                         break;
                     }
@@ -397,7 +423,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
             float *__restrict__ pout = a.partial + ((uint64_t)(i % EP_RING) * a.batch) * a.gpad + cta;
             bool ok = true;
             for (uint32_t s = wg; s < T.nsub; s += EP_GROUP / 32) {   // a warp per sub-tile
-                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars[s], parity, &s_flag[0])) != 0;
+                ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars[s], parity, &s_flag[0], a.wait_ns)) != 0;
                 if (!ok) break;
                 const float *__restrict__ xs = buf + (size_t)s * slot_floats;
                 float acc[SUB];
@@ -428,7 +454,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
             if (sync_any(1u + g, EP_GROUP, s_flag[0])) break;
             if (tg == 0) {
                 asm volatile("fence.acq_rel.gpu;" ::: "memory");   // partials before the count
-                atomicAdd(a.counters + i, 1u);
+                if (i != 0u || cta != a.drop_cta) atomicAdd(a.counters + i, 1u);
             }
         }
 
@@ -436,7 +462,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
         // producer now, so that the copies of the group's next tile run during the exchange ----
         if (stash) {
             // every warp observes the arrival of every sub-tile itself (lane s looks at sub-tile s)
-            for (uint32_t s = lane; s < T.nsub; s += 32u) mbar_wait(&bars[s], parity, &s_flag[0]);
+            for (uint32_t s = lane; s < T.nsub; s += 32u) mbar_wait(&bars[s], parity, &s_flag[0], a.wait_ns);
             __syncwarp();
             for (uint32_t s = 0; s < T.nsub; ++s) {
                 const float *__restrict__ base = buf + (size_t)s * slot_floats + off;
@@ -460,8 +486,8 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
                 const uint64_t t0 = now_ns();
                 uint32_t n = 0u;
                 while (ld_acquire(a.counters + i) < ncta) {
-                    if ((++n & 31u) == 0u) {
-                        if (s_flag[0] != 0u || ld_acquire(a.header) != 0u || now_ns() - t0 > WAIT_LIMIT_NS) {
+                    if ((++n & a.poll_mask) == 0u) {
+                        if (s_flag[0] != 0u || ld_acquire(a.header) != 0u || expired(t0, a.wait_ns)) {
                             s_flag[0] = 1u;
                             break;
                         }
@@ -518,7 +544,7 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
             // parallel), and the warp follows its lanes through __syncwarp.  All of them have
             // landed: the warps that took the margins waited for them.
             if (!stash)
-                for (uint32_t s = lane; s < T.nsub; s += 32u) mbar_wait(&bars[s], parity, &s_flag[0]);
+                for (uint32_t s = lane; s < T.nsub; s += 32u) mbar_wait(&bars[s], parity, &s_flag[0], a.wait_ns);
             __syncwarp();
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (uint32_t s = 0; stash && s < T.nsub; ++s) {
@@ -576,23 +602,11 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
     // Both groups meet here, whether they finished or gave up.
     asm volatile("bar.sync 3, %0;" ::"n"(EP_CONSUMERS) : "memory");
     if (stash && warp == 0) tmem_free_all(tmem_base);   // on every path out of the kernel
-    if (s_flag[0] == 0u) return;
-
-    // ---- a wait ran out: tell the others, let the copies in flight land, leave --------
-    if (tid == 0) {
+    // A wait ran out: tell the host and the other CTAs.  The copies still in flight are the
+    // producer warp's to wait for.
+    if (s_flag[0] != 0u && tid == 0) {
         atomicOr(a.status, QESGD_STATUS_TIMEOUT);
         atomicExch(a.header, 1u);
-    }
-    {
-        const uint64_t t0 = now_ns();
-        while (s_flag[2] == 0u && now_ns() - t0 < 2u * WAIT_LIMIT_NS) __nanosleep(256);
-    }
-    const uint32_t issued = s_flag[1];
-    for (uint32_t b = 0; b < 2u && b < issued; ++b) {
-        const uint32_t last = ((issued - 1u - b) & ~1u) + b;   // last requested tile of buffer b
-        const Tile T = tile_of(a, last);
-        for (uint32_t s = 0; s < T.nsub; ++s)
-            if (!mbar_wait(&full[b * a.nsub_max + s], (last >> 1) & 1u, &s_flag[3])) return;
     }
 }
 
@@ -654,7 +668,8 @@ bool make_map(CUtensorMap *map, const float *X, uint64_t rows, uint64_t d, uint3
 int qesgd_launch_lr_epoch_fused(const float *X, const float *y, uint64_t n_local, uint64_t d,
                                 uint32_t K, uint32_t batch, float lr, float *u, uint64_t u_stride,
                                 float *work, uint64_t work_floats, uint32_t *status, int device,
-                                int sm_count, cudaStream_t stream, int *launched)
+                                int sm_count, uint64_t wait_ns, uint32_t drop_cta, cudaStream_t stream,
+                                int *launched)
 {
     *launched = 0;
     const uint32_t m_full = (uint32_t)(n_local < batch ? n_local : batch);
@@ -683,6 +698,9 @@ int qesgd_launch_lr_epoch_fused(const float *X, const float *y, uint64_t n_local
     a.lr = lr;
     a.u = u; a.u_stride = u_stride;
     a.status = status;
+    a.wait_ns = wait_ns;
+    a.poll_mask = wait_ns < COARSE_TIMER_NS ? 0u : 31u;
+    a.drop_cta = drop_cta;
 
     // shared memory: two tile buffers | coefficients of both groups | barriers | flags
     const size_t smem = (size_t)2 * a.nsub_max * SUB * cols * sizeof(float) + 2 * EP_MAX_M * sizeof(float) +

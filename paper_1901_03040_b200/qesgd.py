@@ -30,6 +30,8 @@ SIGNATURES = {
     "qesgd_create": (_int, [C.POINTER(_vp), _int, _vp]),
     "qesgd_destroy": (_int, [_vp]),
     "qesgd_set_stream": (_int, [_vp, _vp]),
+    "qesgd_set_wait_limit": (_int, [_vp, _u64]),
+    "qesgd_debug_drop_signal": (_int, [_vp, C.c_int64]),
     "qesgd_num_buckets": (_u64, [_u64, _u32]),
     "qesgd_code_bytes": (_u64, [_u64, _u32, _u32]),
     "qesgd_encode": (_int, [_vp, _vp, _vp, _u64, _u32, _u32, _u32, _u32, _f32, _u64, _u32, _u32,
@@ -112,6 +114,12 @@ class Context:
     def set_stream(self, stream):
         self._check(lib.qesgd_set_stream(self._h, C.c_void_p(stream.cuda_stream if stream else 0)))
         self.stream = stream
+
+    def qesgd_set_wait_limit(self, nanoseconds):
+        self._check(lib.qesgd_set_wait_limit(self._h, nanoseconds))
+
+    def qesgd_debug_drop_signal(self, cta):
+        self._check(lib.qesgd_debug_drop_signal(self._h, cta))
 
     # -- worker side ---------------------------------------------------------
     def qesgd_encode(self, local, anchor, d, bucket, s, bits, scale_mode, seed, worker, epoch,

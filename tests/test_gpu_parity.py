@@ -358,6 +358,73 @@ def test_lr_local_epoch_shapes_match_oracle(K, n_local, d, batch):
     assert torch.equal(tu, tu2)
 
 
+# ------------------------------ the local-epoch kernel gives up and recovers ---
+def _epoch_once(c, X, y, n_local, d, K, batch, u0):
+    tu = torch.zeros((K, d), dtype=torch.float32, device="cuda")
+    tu[:] = G.dev(u0)
+    c.qesgd_lr_local_epoch_batch(X, y, n_local, d, K, batch, 0.5, tu, d)
+    return tu, c.qesgd_status()
+
+
+@pytest.mark.parametrize("K,n_local,d,batch", [
+    (2, 96, 8192, 32),       # minibatches stashed in tensor memory between their two uses
+    (3, 200, 4096, 100),     # minibatches that stay in shared memory, odd K
+])
+def test_local_epoch_wait_runs_out_and_the_context_recovers(K, n_local, d, batch):
+    """One CTA never announces its partial margins of the first minibatch (a flag nothing
+    sets), so every CTA's bounded wait for them runs out: the call returns, the status word
+    reports the time-out, nothing faults, and the next call on the same context -- hook off,
+    default limit -- matches the oracle and a fresh context bit for bit."""
+    X, y, _ = synthetic.logistic_problem(K * n_local, d, seed=5 + K)
+    u0 = (0.1 * synthetic.normal_f32(d, 1.0, 22)).astype(np.float32)
+    tX, ty = G.dev(X), G.dev(y)
+    c = qesgd.Context(0, None)
+    c.qesgd_set_wait_limit(3_000_000)              # 3 ms per wait
+    c.qesgd_debug_drop_signal(5)
+    _, status = _epoch_once(c, tX, ty, n_local, d, K, batch, u0)
+    assert status == qesgd.STATUS_TIMEOUT
+    assert c.qesgd_status() == 0                   # reading the status word cleared it
+    c.qesgd_debug_drop_signal(-1)
+    c.qesgd_set_wait_limit(0)                      # back to the default
+    after, status = _epoch_once(c, tX, ty, n_local, d, K, batch, u0)
+    assert status == 0
+    for k in range(K):
+        rows = slice(k * n_local, (k + 1) * n_local)
+        _lr_close(after[k].cpu().numpy(), ref.lr_local_epoch(X[rows], y[rows], batch, 0.5, u0))
+    fresh = qesgd.Context(0, None)
+    want, status = _epoch_once(fresh, tX, ty, n_local, d, K, batch, u0)
+    assert status == 0 and torch.equal(after, want)
+    fresh.close()
+    c.close()
+
+
+def test_local_epoch_with_a_wait_limit_below_the_timer_resolution():
+    """A limit under a microsecond means "look once more, then give up": ordinary latency
+    between CTAs and of the TMA copies exhausts it at whatever point each CTA happens to be,
+    so the give-up path is entered from many places at once.  The call must return either way;
+    a run that happened to need no second look is a complete epoch.  The context recovers."""
+    K, n_local, d, batch = 4, 256, 16384, 32
+    X, y, _ = synthetic.logistic_problem(K * n_local, d, seed=9)
+    u0 = (0.1 * synthetic.normal_f32(d, 1.0, 23)).astype(np.float32)
+    tX, ty = G.dev(X), G.dev(y)
+    want = [ref.lr_local_epoch(X[k * n_local:(k + 1) * n_local], y[k * n_local:(k + 1) * n_local],
+                               batch, 0.5, u0) for k in range(K)]
+    c = qesgd.Context(0, None)
+    for attempt in range(3):
+        c.qesgd_set_wait_limit(100)
+        got, status = _epoch_once(c, tX, ty, n_local, d, K, batch, u0)
+        assert status in (0, qesgd.STATUS_TIMEOUT)
+        if status == 0:
+            for k in range(K):
+                _lr_close(got[k].cpu().numpy(), want[k])
+        c.qesgd_set_wait_limit(0)
+        got, status = _epoch_once(c, tX, ty, n_local, d, K, batch, u0)
+        assert status == 0
+        for k in range(K):
+            _lr_close(got[k].cpu().numpy(), want[k])
+    c.close()
+
+
 # ----------------------------------------------- per-step QESGD (Algorithm 2) ---
 def _gpu_requantize(u, w, zsum, bucket, s, bits, mode, seed, worker, step, fixed_delta=0.0,
                     misalign=0):

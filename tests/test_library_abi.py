@@ -58,6 +58,8 @@ def test_null_context_and_strerror(qesgd):
     assert lib.qesgd_strerror(0) == b"ok"
     assert b"invalid" in lib.qesgd_strerror(qesgd.EINVAL)
     assert lib.qesgd_create(None, 0, None) == qesgd.EINVAL
+    assert lib.qesgd_set_wait_limit(None, 1000) == qesgd.EINVAL
+    assert lib.qesgd_debug_drop_signal(None, 0) == qesgd.EINVAL
 
 
 def test_create_without_a_device_fails_cleanly(qesgd):
