@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the QESGD hot path on B200.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4|c3|c5|c2|c1]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c4|c3|c5|c2|c1|qstep|variance]
   python bench.py --impl reference ...        (the CPU oracle on the host cores)
 
 A step is one pass of the whole path over one batch of synthetic input: all K
@@ -13,7 +13,15 @@ plus 4*d*K for decode-average-apply) divided by the device time of the step.
 
 One JSON line is printed by rank 0.  With N > 1 every rank runs an independent
 replica on its own GPU (the path has no exchange step); the time is the maximum
-over ranks and the value the sum of the work of all ranks over that time.
+over ranks and the value the sum of the work of all ranks over that time.  Started
+plainly with --gpus N (no WORLD_SIZE in the environment) the script starts the N
+ranks itself.
+
+The default line (C4) also carries `sustained` (the same step for most of a second,
+with the SM clock sampled from its first step: the figure under the power cap),
+`cpu_baseline` / `cpu_baseline_all_cores` (the oracle on one thread and on all host
+cores) and `configs`: C1, C2 at d = 2^24, C3 and C5 at three bucket sizes in short
+form, each with its kernels' times, fractions of peak and a parity verdict.
 """
 import argparse
 import json
@@ -50,7 +58,7 @@ def peaks():
     if os.path.exists(path):
         with open(path) as fh:
             return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy bandwidth)"
-    return 6650.0, "fallback (earlier measurement on this pool)"
+    return 6650.0, "fallback (no MEASURED_PEAKS.json beside bench.py)"
 
 
 def ideal_comm_speedup(pull_bits, push_bits=32, full_bits=32):
@@ -74,7 +82,7 @@ class ClockSampler:
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index):
+    def __init__(self, gpu_index, wait_first=False):
         self.tmp = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         self.proc = None
         try:
@@ -84,11 +92,18 @@ class ClockSampler:
                 stdout=self.tmp, stderr=subprocess.DEVNULL)
         except OSError:
             self.proc = None
+        # nvidia-smi needs a few hundred milliseconds before its first line: a region that
+        # wants samples from its very start waits for that line (at most 3 s)
+        t0 = time.time()
+        while wait_first and self.proc is not None and time.time() - t0 < 3.0:
+            if os.path.getsize(self.tmp.name) > 0:
+                break
+            time.sleep(0.02)
 
-    def stop(self):
+    def stop(self, tail=0.25):
         if self.proc is None:
             return None
-        time.sleep(0.25)
+        time.sleep(tail)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -151,6 +166,167 @@ def make_round_inputs(w, device, seed=0):
     return anchor, locs, stride
 
 
+def round_config(w, world):
+    """The `config` object of a round workload; the reference arm prints the same one."""
+    d, K = w["d"], w["K"]
+    return {"workload": w["name"], "d": d, "K": K, "bits": w["bits"], "s": w["s"], "bucket": w["bucket"],
+            "scale_mode": "l2-norm",
+            "l2": "inputs (K*d*4 = %.2f GB) larger than L2; the anchor is re-read from L2 by design"
+                  % (K * d * 4 / 1e9),
+            "parallelism": "replicas only" if world > 1 else "single GPU"}
+
+
+def clocks_bad(clk):
+    if not clk:
+        return False
+    bad = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"} & set(clk["reasons"])
+    stuck = not clk["reasons"] and clk["sm_mhz"] < 0.6 * clk["sm_max_mhz"]
+    return bool(bad) or stuck
+
+
+class RoundBench:
+    """One round workload resident on the device: K locals, the anchor, the parameter, the
+    stream buffers.  step() = qesgd_encode_batch + qesgd_decode_average_apply."""
+
+    def __init__(self, w, device, seed=0):
+        import torch
+        from paper_1901_03040_b200 import qesgd
+        self.w, self.device = w, device
+        self.stream = torch.cuda.Stream(device)
+        self.ctx = qesgd.Context(device.index, self.stream)
+        self.anchor, self.locs, self.stride = make_round_inputs(w, device, seed)
+        self.param = self.anchor.clone()
+        self.codes, self.scales = qesgd.alloc_stream_buffers(w["K"], w["d"], w["bucket"], w["bits"], device)
+        torch.cuda.synchronize()
+
+    def encode(self, epoch):
+        from paper_1901_03040_b200 import qesgd
+        w = self.w
+        self.ctx.qesgd_encode_batch(self.locs, self.stride, self.param, w["d"], w["K"], w["bucket"], w["s"],
+                                    w["bits"], qesgd.SCALE_NORM, 2024, 0, epoch, self.codes,
+                                    self.codes.stride(0), self.scales, self.scales.stride(0))
+
+    def apply(self):
+        w = self.w
+        self.ctx.qesgd_decode_average_apply(self.param, w["d"], w["K"], self.codes, self.codes.stride(0),
+                                            self.scales, self.scales.stride(0), w["bucket"], w["s"], w["bits"])
+
+    def step(self, epoch):
+        self.encode(epoch)
+        self.apply()
+
+    def timed(self, first_epoch, steps, sampler=None, sampler_tail=0.25, barrier=None):
+        """`steps` steps between one event pair, per-kernel events inside.  Returns
+        (total ms, encode ms per step, apply ms per step, clocks, launches)."""
+        import torch
+        launches0 = self.ctx.qesgd_launch_count()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+        t_begin = torch.cuda.Event(enable_timing=True)
+        t_end = torch.cuda.Event(enable_timing=True)
+        t_begin.record(self.stream)
+        for i in range(steps):
+            ev[i][0].record(self.stream)
+            self.encode(first_epoch + i)
+            ev[i][1].record(self.stream)
+            self.apply()
+            ev[i][2].record(self.stream)
+        t_end.record(self.stream)
+        if barrier is not None:
+            barrier()
+        else:
+            torch.cuda.synchronize()
+        clk = sampler.stop(sampler_tail) if sampler else None
+        return (t_begin.elapsed_time(t_end), [e[0].elapsed_time(e[1]) for e in ev],
+                [e[1].elapsed_time(e[2]) for e in ev], clk, self.ctx.qesgd_launch_count() - launches0)
+
+    def kernel_records(self, enc_ms, daa_ms, peak):
+        w = self.w
+        d, K = w["d"], w["K"]
+        enc_bytes, daa_bytes = round_bytes(w)
+        out = {}
+        for name, ms, nbytes, elems in (("encode_batch", enc_ms, enc_bytes, d * K),
+                                        ("decode_average_apply", daa_ms, daa_bytes, d)):
+            avg = statistics.mean(ms)
+            gbs = nbytes / (avg * 1e-3) / 1e9
+            out[name] = {"avg_ms": avg, "min_ms": min(ms), "algorithmic_bytes": nbytes, "hbm_gbs": gbs,
+                         "frac_of_peak": gbs / peak, "frac_of_8000": gbs / 8000.0,
+                         "fp32_equiv_gbs": 4.0 * d * K / (avg * 1e-3) / 1e9,
+                         "elements_per_s": elems / (avg * 1e-3)}
+        return out
+
+    def close(self):
+        import torch
+        self.ctx.close()
+        del self.anchor, self.locs, self.param, self.codes, self.scales
+        torch.cuda.empty_cache()
+
+
+def sampled_bucket_parity(rb, n_buckets, seed=1):
+    """One untimed round from param = anchor, then the CPU oracle on `n_buckets` buckets drawn
+    over the whole vector (plus the first two, the middle one and the last two): a bucket's
+    codes and scale depend only on its own elements and their global indices, so each sampled
+    bucket is checked exactly; the applied parameter within 1e-6."""
+    import numpy as np
+    import torch
+    from oracle import qesgd_ref as ref
+    from paper_1901_03040_b200 import qesgd
+    w = rb.w
+    d, K, bits, s, B = w["d"], w["K"], w["bits"], w["s"], w["bucket"]
+    rb.param.copy_(rb.anchor)
+    torch.cuda.synchronize()          # the copy ran on torch's stream, the library runs on its own
+    rb.encode(7)
+    rb.apply()
+    status = rb.ctx.qesgd_status()
+    nb = qesgd.num_buckets(d, B)
+    rng = np.random.default_rng(seed)
+    picks = sorted(set(rng.integers(0, nb, size=n_buckets).tolist())
+                   | {0, min(1, nb - 1), nb // 2, max(0, nb - 2), nb - 1})
+    bpb = B * bits // 8
+    idx = torch.tensor(picks, device=rb.device)
+    g_scales = rb.scales[:, idx].cpu().numpy()
+    byte_idx = (idx[:, None] * bpb + torch.arange(bpb, device=rb.device)[None, :]).reshape(-1)
+    g_codes = rb.codes[:, byte_idx].cpu().numpy().reshape(K, len(picks), bpb)
+    elem_idx = (idx[:, None] * B + torch.arange(B, device=rb.device)[None, :]).reshape(-1).clamp_(max=d - 1)
+    h_anchor = rb.anchor[elem_idx].cpu().numpy().reshape(len(picks), B)
+    h_param = rb.param[elem_idx].cpu().numpy().reshape(len(picks), B)
+    h_locs = rb.locs[:, elem_idx].cpu().numpy().reshape(K, len(picks), B)
+    bad = {"codes": 0, "scales": 0, "param": 0}
+    for n, j in enumerate(picks):
+        lo, hi = j * B, min((j + 1) * B, d)
+        m = hi - lo
+        r_codes, r_scales = [], []
+        for k in range(K):
+            c, sc, _ = ref.encode(h_locs[k, n, :m], h_anchor[n, :m], B, s, bits, ref.SCALE_NORM, 2024, k, 7,
+                                  i0=lo)
+            r_codes.append(c)
+            r_scales.append(sc)
+            bad["codes"] += int((g_codes[k, n].view(np.uint32) != c).any())
+            bad["scales"] += int(g_scales[k, n].view(np.uint32) != sc.view(np.uint32)[0])
+        r_scales = np.stack(r_scales)
+        want = ref.decode_average_apply(h_anchor[n, :m], np.stack(r_codes), r_scales, B, s, bits)
+        tol = 1e-6 * np.maximum(np.abs(want), r_scales.max())
+        bad["param"] += int((np.abs(h_param[n, :m].astype(np.float64) - want) > tol).any())
+    return {"buckets_checked": len(picks), "workers": K, "codes_bit_exact": bad["codes"] == 0,
+            "scales_bit_exact": bad["scales"] == 0, "param_within_1e-6": bad["param"] == 0,
+            "status_flags": status}
+
+
+def sustained_leg(rb, first_epoch, ms_per_step, peak, gpu_index, seconds=0.8):
+    """The same step repeated for `seconds`: long enough for the power cap to settle the SM
+    clock, with clock samples taken from the first step on.  time x MHz makes runs at different
+    clocks comparable (the codec kernels are bound by instruction issue)."""
+    steps = int(min(20000, max(50, seconds * 1e3 / max(ms_per_step, 1e-3))))
+    sampler = ClockSampler(gpu_index, wait_first=True)
+    total_ms, enc_ms, daa_ms, clk, _ = rb.timed(first_epoch, steps, sampler, sampler_tail=0.03)
+    rec = {"steps": steps, "seconds": total_ms * 1e-3, "ms_per_step": total_ms / steps,
+           "value": 2.0 * 4.0 * rb.w["d"] * rb.w["K"] * steps / (total_ms * 1e-3) / 1e9, "unit": UNIT,
+           "kernels": rb.kernel_records(enc_ms, daa_ms, peak), "clocks": clk}
+    if clk:
+        for name in rec["kernels"]:
+            rec["kernels"][name]["ms_x_mhz"] = rec["kernels"][name]["avg_ms"] * clk["sm_mhz"]
+    return rec, steps
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -167,37 +343,41 @@ def run_ours(args):
             if os.path.exists(lib_build.LIB) and not lib_build._stale(lib_build.LIB, sources):
                 break
             time.sleep(0.5)
-    from paper_1901_03040_b200 import qesgd
+    from paper_1901_03040_b200 import qesgd  # noqa: F401  (raises if the library is missing)
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py: no CUDA device; the CUDA path has no fallback")
+    if local >= torch.cuda.device_count():
+        raise SystemExit(f"bench.py: rank {rank} wants cuda:{local} but only "
+                         f"{torch.cuda.device_count()} device(s) are visible")
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=device)
     if args.workload == "c2":
-        return run_c2(args, device, world, rank)
-    if args.workload == "c1":
-        return run_c1(args, device, world, rank)
-    if args.workload == "qstep":
-        return run_qstep(args, device, world, rank)
+        line = run_c2(args, device, world, rank)
+    elif args.workload == "c1":
+        line = run_c1(args, device, world, rank)
+    elif args.workload == "qstep":
+        line = run_qstep(args, device, world, rank)
+    elif args.workload == "variance":
+        line = run_variance(args, device, world, rank)
+    else:
+        line = run_round(args, device, world, rank, local)
+    if rank == 0:
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def run_round(args, device, world, rank, local):
+    import torch
+    import torch.distributed as dist
     w = dict(WORKLOADS[args.workload])
     if args.bucket:
         w["bucket"] = args.bucket
-    d, K, bits, s, B = w["d"], w["K"], w["bits"], w["s"], w["bucket"]
-
-    stream = torch.cuda.Stream(device)
-    ctx = qesgd.Context(local, stream)
-    anchor, locs, stride = make_round_inputs(w, device)
-    param = anchor.clone()
-    codes, scales = qesgd.alloc_stream_buffers(K, d, B, bits, device)
-    torch.cuda.synchronize()
-
-    def step(epoch):
-        ctx.qesgd_encode_batch(locs, stride, param, d, K, B, s, bits, qesgd.SCALE_NORM, 2024, 0,
-                               epoch, codes, codes.stride(0), scales, scales.stride(0))
-        ctx.qesgd_decode_average_apply(param, d, K, codes, codes.stride(0), scales,
-                                       scales.stride(0), B, s, bits)
+    d, K = w["d"], w["K"]
+    rb = RoundBench(w, device)
 
     def barrier():
         torch.cuda.synchronize()
@@ -206,73 +386,56 @@ def run_ours(args):
         torch.cuda.synchronize()
 
     for i in range(args.warmup):
-        step(i)
+        rb.step(i)
     barrier()
-    def timed_region(first_epoch):
-        launches0 = ctx.qesgd_launch_count()
-        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-        sampler = ClockSampler(local) if rank == 0 else None
-        t_begin = torch.cuda.Event(enable_timing=True)
-        t_end = torch.cuda.Event(enable_timing=True)
-        t_begin.record(stream)
-        for i in range(args.steps):
-            ev[i][0].record(stream)
-            ctx.qesgd_encode_batch(locs, stride, param, d, K, B, s, bits, qesgd.SCALE_NORM, 2024, 0,
-                                   first_epoch + i, codes, codes.stride(0), scales, scales.stride(0))
-            ev[i][1].record(stream)
-            ctx.qesgd_decode_average_apply(param, d, K, codes, codes.stride(0), scales,
-                                           scales.stride(0), B, s, bits)
-            ev[i][2].record(stream)
-        t_end.record(stream)
-        barrier()
-        clk = sampler.stop() if sampler else None
-        return (t_begin.elapsed_time(t_end), [e[0].elapsed_time(e[1]) for e in ev],
-                [e[1].elapsed_time(e[2]) for e in ev], clk, ctx.qesgd_launch_count() - launches0)
-
-    def clocks_bad(clk):
-        if not clk:
-            return False
-        bad = {"hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown"} & set(clk["reasons"])
-        stuck = not clk["reasons"] and clk["sm_mhz"] < 0.6 * clk["sm_max_mhz"]
-        return bool(bad) or stuck
-
-    total_ms, enc_ms, daa_ms, clocks, launches = timed_region(args.warmup)
+    sampler = ClockSampler(local) if rank == 0 else None
+    total_ms, enc_ms, daa_ms, clocks, launches = rb.timed(args.warmup, args.steps, sampler, barrier=barrier)
     remeasured = False
     again = 1.0 if (rank == 0 and clocks_bad(clocks)) else 0.0
     _, again = aggregate_over_ranks(0.0, again, world, device, world > 1)
     if again > 0.0:       # thermal or hardware slowdown, or clocks pinned low: measure once more
         remeasured = True
-        total_ms, enc_ms, daa_ms, clocks, launches = timed_region(args.warmup + args.steps)
+        sampler = ClockSampler(local) if rank == 0 else None
+        total_ms, enc_ms, daa_ms, clocks, launches = rb.timed(args.warmup + args.steps, args.steps, sampler,
+                                                              barrier=barrier)
     if clocks is not None:
         clocks["remeasured"] = remeasured
         clocks["rejected"] = clocks_bad(clocks)
-    status = ctx.qesgd_status()
+    status = rb.ctx.qesgd_status()
 
     fp32_equiv_bytes = 2.0 * 4.0 * d * K * args.steps
     ms_all, units_all = aggregate_over_ranks(total_ms, fp32_equiv_bytes, world, device, world > 1)
     value = units_all / (ms_all * 1e-3) / 1e9
+    peak, peak_src = peaks()
+    kernels = rb.kernel_records(enc_ms, daa_ms, peak)
+
+    # ---- the same step for most of a second: the figure under the power cap ---------------
+    sustained = None
+    if rank == 0 and world == 1 and not args.no_sustained:
+        sustained, used = sustained_leg(rb, args.warmup + 2 * args.steps, ms_all / args.steps, peak, local,
+                                        args.sustained_seconds)
 
     # ---- end to end: host buffers in, host result out, through the same calls -----------
     e2e = None
-    cpu_baseline = None
-    parity = None
+    cpu_baseline = cpu_all = parity = None
     if not args.no_e2e:
+        stride = rb.stride
         h_locs = torch.empty((K, stride), dtype=torch.float32, pin_memory=True)
-        h_locs.copy_(locs)
+        h_locs.copy_(rb.locs)
         h_param = torch.empty((d,), dtype=torch.float32, pin_memory=True)
         torch.cuda.synchronize()
         e2e_steps = max(1, min(args.steps, 3))
         e_begin = torch.cuda.Event(enable_timing=True)
         e_end = torch.cuda.Event(enable_timing=True)
-        with torch.cuda.stream(stream):
+        with torch.cuda.stream(rb.stream):
             for i in range(1 + e2e_steps):
                 if i == 1:
                     barrier()
-                    e_begin.record(stream)
-                locs.copy_(h_locs, non_blocking=True)
-                step(1000 + i)
-                h_param.copy_(param, non_blocking=True)
-            e_end.record(stream)
+                    e_begin.record(rb.stream)
+                rb.locs.copy_(h_locs, non_blocking=True)
+                rb.step(100000 + i)
+                h_param.copy_(rb.param, non_blocking=True)
+            e_end.record(rb.stream)
             barrier()
         e2e_ms, e2e_units = aggregate_over_ranks(e_begin.elapsed_time(e_end),
                                                  2.0 * 4.0 * d * K * e2e_steps, world, device,
@@ -285,48 +448,100 @@ def run_ours(args):
 
     # ---- the CPU oracle on a bounded sample of the same inputs, with a parity check -------
     if rank == 0 and world == 1 and not args.no_cpu:
-        cpu_baseline, parity = oracle_sample(ctx, w, locs, stride, anchor, device,
-                                             args.cpu_sample_elems)
+        cpu_baseline, cpu_all, parity = oracle_sample(rb.ctx, w, rb.locs, rb.stride, rb.anchor, device,
+                                                      args.cpu_sample_elems)
 
-    peak, peak_src = peaks()
-    enc_bytes, daa_bytes = round_bytes(w)
-    enc_avg = statistics.mean(enc_ms)
-    daa_avg = statistics.mean(daa_ms)
-    enc_gbs = enc_bytes / (enc_avg * 1e-3) / 1e9
-    daa_gbs = daa_bytes / (daa_avg * 1e-3) / 1e9
     traffic = load_traffic("encode", args.workload)
+    enc = kernels["encode_batch"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_all / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": w["name"], "d": d, "K": K, "bits": bits, "s": s, "bucket": B,
-                   "scale_mode": "l2-norm", "l2": "inputs (K*d*4 = %.2f GB) larger than L2; the "
-                   "anchor is re-read from L2 by design" % (K * d * 4 / 1e9),
-                   "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "config": round_config(w, world),
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "qesgd_encode_kernel (encode_batch, K workers)",
-                     "achieved": enc_gbs, "peak": peak, "unit": "GB/s", "frac": enc_gbs / peak,
+                     "achieved": enc["hbm_gbs"], "peak": peak, "unit": "GB/s", "frac": enc["frac_of_peak"],
                      "traffic": traffic, "peak_source": peak_src,
-                     "algorithmic_bytes_per_launch": enc_bytes, "avg_launch_ms": enc_avg},
-        "kernels": {
-            "encode_batch": {"avg_ms": enc_avg, "min_ms": min(enc_ms), "hbm_gbs": enc_gbs,
-                             "frac_of_peak": enc_gbs / peak, "frac_of_8000": enc_gbs / 8000.0,
-                             "fp32_equiv_gbs": 4.0 * d * K / (enc_avg * 1e-3) / 1e9,
-                             "elements_per_s": d * K / (enc_avg * 1e-3)},
-            "decode_average_apply": {"avg_ms": daa_avg, "min_ms": min(daa_ms), "hbm_gbs": daa_gbs,
-                                     "frac_of_peak": daa_gbs / peak, "frac_of_8000": daa_gbs / 8000.0,
-                                     "fp32_equiv_gbs": 4.0 * d * K / (daa_avg * 1e-3) / 1e9,
-                                     "elements_per_s": d / (daa_avg * 1e-3)}},
+                     "algorithmic_bytes_per_launch": enc["algorithmic_bytes"], "avg_launch_ms": enc["avg_ms"]},
+        "kernels": kernels,
         "status_flags": status,
         "clocks": clocks,
+        "sustained": sustained,
         "e2e": e2e,
         "cpu_baseline": cpu_baseline,
+        "cpu_baseline_all_cores": cpu_all,
         "parity_on_sample": parity,
     }
-    if rank == 0:
-        print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+    rb.close()
+    # ---- the other configurations, each with its kernels' times and a parity verdict ------
+    if rank == 0 and world == 1 and args.workload == "c4" and not args.no_configs:
+        line["configs"] = other_configs(args, device, peak)
+    return line
+
+
+def other_configs(args, device, peak):
+    """C1, C2 (d = 2^24), C3 and C5 (three bucket sizes) in short form: per hot kernel its mean
+    time, algorithmic bytes and fraction of the measured and of the nominal 8000 GB/s peak, and
+    a parity verdict from the CPU oracle on a sample.  20 timed steps each after 3 warm-ups."""
+    import copy
+    import torch
+    out = {}
+    sub = copy.copy(args)
+    sub.steps, sub.warmup, sub.d, sub.scale_mode = 20, 3, 0, "norm"
+    t0 = time.time()
+
+    def short(kernels):
+        keep = ("avg_ms", "min_ms", "algorithmic_bytes", "hbm_gbs", "frac_of_peak", "frac_of_8000")
+        return {k: {f: v[f] for f in keep if f in v} for k, v in kernels.items()}
+
+    try:
+        c1 = run_c1(sub, device, 1, 0)
+        out["c1"] = {"workload": c1["config"]["workload"], "round_ms": c1["value"],
+                     "kernels": c1["kernels"], "parity": c1["first_round"].get("oracle"),
+                     "loss_before": c1["loss_before"], "loss_after_first_round": c1["loss_after_first_rounds"][0],
+                     "clocks": c1.get("clocks")}
+    except Exception as exc:  # noqa: BLE001  (one configuration must not take the bench line down)
+        out["c1"] = {"error": repr(exc)}
+    torch.cuda.empty_cache()
+    try:
+        sub.steps = 200
+        c2 = run_c2(sub, device, 1, 0)
+        out["c2"] = {"workload": c2["config"]["workload"], "d": c2["config"]["d"],
+                     "launch": c2["config"]["launch"], "kernels": short(c2["kernels"]),
+                     "parity": c2["parity_on_sample"], "clocks": c2["clocks"]}
+    except Exception as exc:  # noqa: BLE001
+        out["c2"] = {"error": repr(exc)}
+    torch.cuda.empty_cache()
+    sub.steps = 20
+    todo = [("c3", dict(WORKLOADS["c3"]), 256)]
+    for bucket in (128, 512, 4096):
+        w = dict(WORKLOADS["c5"])
+        w["bucket"] = bucket
+        todo.append((f"c5_bucket{bucket}", w, 256 if bucket < 4096 else 64))
+    for name, w, n_buckets in todo:
+        try:
+            need = w["d"] * (w["K"] * 4.6 + 8.5)
+            free, _ = torch.cuda.mem_get_info()
+            if free < need * 1.1:
+                out[name] = {"skipped": f"needs {need / 1e9:.0f} GB of device memory, {free / 1e9:.0f} GB free"}
+                continue
+            rb = RoundBench(w, device, seed=len(name))
+            for i in range(3):
+                rb.step(i)
+            torch.cuda.synchronize()
+            sampler = ClockSampler(device.index or 0, wait_first=True)
+            _, enc_ms, daa_ms, clk, _ = rb.timed(3, sub.steps, sampler, sampler_tail=0.03)
+            rec = {"workload": w["name"], "bucket": w["bucket"],
+                   "kernels": short(rb.kernel_records(enc_ms, daa_ms, peak)), "clocks": clk}
+            if not args.no_cpu:
+                rec["parity"] = sampled_bucket_parity(rb, n_buckets)
+            out[name] = rec
+            rb.close()
+        except Exception as exc:  # noqa: BLE001
+            out[name] = {"error": repr(exc)}
+        torch.cuda.empty_cache()
+    out["seconds"] = time.time() - t0
+    return out
 
 
 def load_traffic(kernel, workload):
@@ -355,12 +570,46 @@ def load_traffic(kernel, workload):
         return None
 
 
+def oracle_round_on_slices(h_loc, h_anchor, w, epoch, threads):
+    """The oracle's round (encode of every worker, then decode-average-apply) on host arrays.
+    With threads > 1 the vector is cut into bucket ranges, one per thread: buckets are
+    independent, the oracle takes a slice with its global offset, and its C calls release the
+    interpreter lock.  Returns (codes [K, words], scales [K, nb], new parameter)."""
+    import numpy as np
+    from concurrent.futures import ThreadPoolExecutor
+    from oracle import qesgd_ref as ref
+    K, n = h_loc.shape
+    bits, s, B = w["bits"], w["s"], w["bucket"]
+    nb = (n + B - 1) // B
+    cuts = [min(nb, (nb * t) // threads) for t in range(threads + 1)]
+    ranges = [(cuts[t] * B, min(n, cuts[t + 1] * B)) for t in range(threads) if cuts[t + 1] > cuts[t]]
+
+    def work(r):
+        lo, hi = r
+        cs, ss = [], []
+        for k in range(K):
+            c, sc, _ = ref.encode(h_loc[k, lo:hi], h_anchor[lo:hi], B, s, bits, ref.SCALE_NORM, 2024, k, epoch,
+                                  i0=lo)
+            cs.append(c)
+            ss.append(sc)
+        cs, ss = np.stack(cs), np.stack(ss)
+        return cs, ss, ref.decode_average_apply(h_anchor[lo:hi], cs, ss, B, s, bits)
+
+    if len(ranges) == 1:
+        parts = [work(ranges[0])]
+    else:
+        with ThreadPoolExecutor(max_workers=len(ranges)) as pool:
+            parts = list(pool.map(work, ranges))
+    return (np.concatenate([p[0] for p in parts], axis=1), np.concatenate([p[1] for p in parts], axis=1),
+            np.concatenate([p[2] for p in parts]))
+
+
 def oracle_sample(ctx, w, locs, stride, anchor, device, sample_elems):
-    """Time the CPU oracle (as it stands, one thread) on the first `sample_elems` elements of
-    every worker and compare the GPU's output on the same slice with it."""
+    """Time the CPU oracle (as it stands) on the first `sample_elems` elements of every worker,
+    once on one thread and once with the bucket ranges spread over all host cores, and compare
+    the GPU's output on the same slice with it."""
     import numpy as np
     import torch
-    from oracle import qesgd_ref as ref
     from paper_1901_03040_b200 import qesgd
     d, K, bits, s, B = w["d"], w["K"], w["bits"], w["s"], w["bucket"]
     n = min(d, sample_elems) // B * B          # whole buckets only
@@ -378,24 +627,28 @@ def oracle_sample(ctx, w, locs, stride, anchor, device, sample_elems):
     g_scales = scales[:, :nb].cpu().numpy()
     g_param = param[:n].cpu().numpy()
     t0 = time.perf_counter()
-    r_codes, r_scales = [], []
-    for k in range(K):
-        c, sc, _ = ref.encode(h_loc[k], h_anchor, B, s, bits, ref.SCALE_NORM, 2024, k, 7)
-        r_codes.append(c)
-        r_scales.append(sc)
-    r_codes, r_scales = np.stack(r_codes), np.stack(r_scales)
-    r_param = ref.decode_average_apply(h_anchor, r_codes, r_scales, B, s, bits)
+    r_codes, r_scales, r_param = oracle_round_on_slices(h_loc, h_anchor, w, 7, 1)
     dt = time.perf_counter() - t0
+    cores = max(1, len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else (os.cpu_count() or 1))
+    t0 = time.perf_counter()
+    a_codes, a_scales, a_param = oracle_round_on_slices(h_loc, h_anchor, w, 7, cores)
+    dt_all = time.perf_counter() - t0
     tol = 1e-6 * np.maximum(np.abs(r_param), np.repeat(r_scales.max(0), B)[:n])
     parity = {"codes_bit_exact": bool((g_codes == r_codes).all()),
               "scales_bit_exact": bool((g_scales.view(np.uint32) == r_scales.view(np.uint32)).all()),
               "param_within_1e-6": bool((np.abs(g_param.astype(np.float64) - r_param) <= tol).all()),
+              "all_cores_run_equals_one_core_run": bool((a_codes == r_codes).all() and (a_param == r_param).all()
+                                                        and (a_scales == r_scales).all()),
               "elements": int(n), "workers": int(K)}
+    what = (f"first {n} elements of each of the {K} workers: encode of every worker, then "
+            f"decode-average-apply")
     cpu = {"value": 2.0 * 4.0 * n * K / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-           "sample": f"first {n} elements of each of the {K} workers: encode of every worker, then "
-                     f"decode-average-apply ({dt:.1f} s of CPU time)",
-           "seconds": dt}
-    return cpu, parity
+           "sample": f"{what} ({dt:.1f} s of CPU time)", "seconds": dt,
+           "elements_per_s": n * K / dt}
+    cpu_all = {"value": 2.0 * 4.0 * n * K / dt_all / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+               "sample": f"{what}; bucket ranges spread over {cores} threads ({dt_all:.1f} s)",
+               "seconds": dt_all, "elements_per_s": n * K / dt_all}
+    return cpu, cpu_all, parity
 
 
 # --------------------------------------------------- other workloads (own arm) ---
@@ -419,7 +672,7 @@ def run_c2(args, device, world, rank):
     results = {}
     t_total = 0.0
     graph_launches = 0      # kernel nodes replayed inside the timed regions
-    sampler = ClockSampler(device.index) if rank == 0 else None
+    sampler = ClockSampler(device.index, wait_first=True) if rank == 0 else None
     for bits, s in variants:
         for kind in ("encode", "decode"):
             def call(i):
@@ -488,8 +741,41 @@ def run_c2(args, device, world, rank):
                          "frac": enc["frac_of_peak"], "traffic": load_traffic("encode", "c2"),
                          "peak_source": peak_src},
             "kernels": results, "clocks": clocks}
-    if rank == 0:
-        print(json.dumps(line))
+    for rec in results.values():
+        rec["frac_of_8000"] = rec["hbm_gbs"] / 8000.0
+        rec["algorithmic_bytes"] = rec["hbm_gbs"] * 1e9 * rec["avg_ms"] * 1e-3
+    if rank == 0 and world == 1 and not args.no_cpu:
+        line["parity_on_sample"] = c2_parity(ctx, zs[0], d, B, mode, variants, device)
+    else:
+        line["parity_on_sample"] = None
+    ctx.close()
+    return line
+
+
+def c2_parity(ctx, z, d, B, mode, variants, device, n=1 << 21):
+    """Encode and decode of the first n elements (whole buckets) against the CPU oracle, all
+    three code widths: codes, scales and decoded values bit for bit."""
+    import numpy as np
+    import torch
+    from oracle import qesgd_ref as ref
+    from paper_1901_03040_b200 import qesgd
+    n = min(n, d) // B * B
+    h = z[:n].cpu().numpy()
+    ok = {}
+    for bits, s in variants:
+        codes, scales = qesgd.alloc_stream_buffers(1, n, B, bits, device)
+        out = torch.empty(n, dtype=torch.float32, device=device)
+        ctx.qesgd_encode(z, None, n, B, s, bits, mode, 1, 0, 3, codes, scales, fixed_delta=3e-3 / s)
+        ctx.qesgd_decode(codes, scales, n, B, s, bits, out)
+        torch.cuda.synchronize()
+        r_codes, r_scales, _ = ref.encode(h, None, B, s, bits, mode, 1, 0, 3, fixed_delta=3e-3 / s)
+        r_out = ref.decode(r_codes, r_scales, n, B, s, bits)
+        g_codes = codes.view(-1)[:n * bits // 8].cpu().numpy().view(np.uint32)
+        g_scales = scales.view(-1)[:n // B].cpu().numpy()
+        ok[f"{bits}bit"] = bool((g_codes == r_codes).all()
+                                and (g_scales.view(np.uint32) == r_scales.view(np.uint32)).all()
+                                and (out.cpu().numpy().view(np.uint32) == r_out.view(np.uint32)).all())
+    return {"elements": int(n), "codes_scales_decoded_bit_exact": ok}
 
 
 def run_qstep(args, device, world, rank):
@@ -538,8 +824,8 @@ def run_qstep(args, device, world, rank):
                          "peak": peak, "unit": "GB/s", "frac": gbs / peak, "traffic": None,
                          "peak_source": peak_src, "algorithmic_bytes_per_launch": nbytes},
             "status_flags": ctx.qesgd_status(), "clocks": clocks}
-    if rank == 0:
-        print(json.dumps(line))
+    ctx.close()
+    return line
 
 
 def run_c1(args, device, world, rank):
@@ -619,8 +905,90 @@ def run_c1(args, device, world, rank):
                                 "cores": 1, "kind": "oracle",
                                 "sample": "the whole of round 1: four local epochs, encode of the four "
                                           "workers, decode-average-apply"}
-    if rank == 0:
-        print(json.dumps(line))
+    ctx.close()
+    return line
+
+
+def quantisation_variance(ctx, v, bucket, s, bits, draws, seed=5):
+    """Monte-Carlo E||Q(v) - v||^2 of the library's quantiser (encode with anchor = NULL and
+    the bucket's L2 norm as scale, then decode) over `draws` epochs of draws, beside Lemma 1's
+    closed form sum_i delta_b^2 p_i (1 - p_i), p_i the fractional part of |v_i| / delta_b and
+    delta_b = fl32(scale_b / s) the decoder's grid spacing.  v is a device vector; the sums are
+    taken in fp64 on the device (measurement only: the path itself is the two library calls)."""
+    import torch
+    from paper_1901_03040_b200 import qesgd
+    d = v.numel()
+    codes, scales = qesgd.alloc_stream_buffers(1, d, bucket, bits, v.device)
+    out = torch.empty(d, dtype=torch.float32, device=v.device)
+    acc = 0.0
+    for e in range(draws):
+        ctx.qesgd_encode(v, None, d, bucket, s, bits, qesgd.SCALE_NORM, seed, 0, e, codes, scales)
+        ctx.qesgd_decode(codes, scales, d, bucket, s, bits, out)
+        (ctx.stream or torch.cuda.current_stream()).synchronize()
+        acc += float(((out.double() - v.double()) ** 2).sum().item())
+    nb = qesgd.num_buckets(d, bucket)
+    delta = (scales.view(-1)[:nb] / float(s)).double()              # fl32(scale/s), then exact
+    delta_e = delta.repeat_interleave(bucket)[:d]
+    r = torch.where(delta_e > 0, v.double().abs() / delta_e.clamp_min(1e-300), torch.zeros_like(delta_e))
+    p = r - torch.floor(r)
+    closed = float((delta_e ** 2 * p * (1.0 - p)).sum().item())
+    bound = float((delta_e ** 2).sum().item()) / 4.0              # d * delta^2 / 4 (proof of Theorem 1)
+    return {"monte_carlo": acc / draws, "closed_form": closed, "bound_d_delta2_over_4": bound,
+            "norm2": float((v.double() ** 2).sum().item()), "draws": draws}
+
+
+def run_variance(args, device, world, rank):
+    """Gradient compression (the QSGD baseline of Sec. 5: delta = ||g||) against compression of the
+    epoch delta (QESGD, Sec. 2.2) on the C1 logistic problem, same code width and bucket: the
+    quantisation noise E||Q(v) - v||^2 of a minibatch gradient g and of a local-epoch delta
+    z = u - w_t, each against Lemma 1's closed form, and what either scheme adds to the
+    parameter per epoch: QSGD quantises every one of the epoch's steps (noise lr^2 * Var per
+    step), QESGD quantises once per epoch."""
+    import torch
+    from paper_1901_03040_b200 import qesgd, synthetic
+    n, d, K, batch, lr, B, s, bits = 8192, 65536, 4, 64, 0.1, 512, 127, 8
+    if args.d:
+        d = args.d
+    draws = max(8, min(args.steps, 256))
+    stream = torch.cuda.Stream(device)
+    ctx = qesgd.Context(device.index, stream)
+    X, y, _ = synthetic.logistic_problem(n, d, seed=0)
+    tX, ty = torch.from_numpy(X).to(device), torch.from_numpy(y).to(device)
+    n_local = n // K
+    w = torch.zeros(d, dtype=torch.float32, device=device)
+    g = torch.empty(d, dtype=torch.float32, device=device)
+    u = torch.zeros((1, d), dtype=torch.float32, device=device)
+    torch.cuda.synchronize()
+    t0 = time.time()
+    ctx.qesgd_lr_gradient(tX[:batch], ty[:batch], batch, d, w, g)
+    ctx.qesgd_lr_local_epoch_batch(tX, ty, n_local, d, 1, batch, lr, u, d)
+    stream.synchronize()
+    z = (u[0] - w).contiguous()
+    res = {}
+    for bits_, s_ in ((8, 127), (4, 7), (2, 1)):
+        rg = quantisation_variance(ctx, g, B, s_, bits_, draws)
+        rz = quantisation_variance(ctx, z, B, s_, bits_, draws)
+        steps = n_local // batch
+        res[f"{bits_}bit"] = {
+            "gradient": rg, "epoch_delta": rz,
+            "relative_noise": {"gradient": rg["monte_carlo"] / rg["norm2"],
+                               "epoch_delta": rz["monte_carlo"] / rz["norm2"]},
+            "parameter_noise_per_epoch": {"qsgd_every_step": steps * lr * lr * rg["monte_carlo"],
+                                          "qesgd_once": rz["monte_carlo"]},
+            "monte_carlo_over_closed_form": {"gradient": rg["monte_carlo"] / rg["closed_form"],
+                                             "epoch_delta": rz["monte_carlo"] / rz["closed_form"]}}
+    dt = time.time() - t0
+    line = {"metric": "quantisation noise E||Q(v)-v||^2, gradient vs epoch delta", "value": dt, "unit": "s",
+            "n_gpus": world, "steps": draws, "warmup": 0, "ms_per_step": dt * 1e3 / draws,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": "variance of Q(g) against Q(z) on the C1 logistic problem (worker 0, "
+                                   "w = 0, minibatch 64, lr 0.1, bucket 512, L2-norm scale)", "d": d,
+                       "draws": draws},
+            "gpu_launches": int(ctx.qesgd_launch_count()), "results": res,
+            "status_flags": ctx.qesgd_status()}
+    ctx.close()
+    return line
 
 
 def c1_first_round(args, rank, world, X, y, u, codes, scales, param, loss, shape):
@@ -665,7 +1033,7 @@ def run_reference(args):
     """The CPU oracle, as it stands, on the host cores: each step runs the whole path on a
     bounded sample of the workload (first elements of every worker)."""
     world, rank, _ = dist_info()
-    if rank != 0:
+    if rank != 0:          # under torchrun rank 0 alone runs the oracle; the others leave
         return
     import numpy as np
     from oracle import qesgd_ref as ref
@@ -701,10 +1069,9 @@ def run_reference(args):
     sample = f"first {n} elements of each of the {K} workers per step (one thread)"
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 / args.steps,
-            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64/f32",
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
-            "config": {"workload": w["name"], "d": d, "K": K, "bits": bits, "s": s, "bucket": B,
-                       "sample": sample},
+            "config": round_config(w, 1),
             "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
                              "sample": sample},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -712,29 +1079,58 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def main():
+def torchrun_command(gpus, argv, port=None):
+    """The command that runs this file as `gpus` ranks on this node, one per GPU."""
+    if port is None:
+        import socket
+        with socket.socket() as sock:
+            sock.bind(("127.0.0.1", 0))
+            port = sock.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={gpus}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
+def main(argv=None):
+    argv = sys.argv[1:] if argv is None else argv
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--workload", choices=["c4", "c3", "c5", "c2", "c1", "qstep"], default="c4")
+    ap.add_argument("--workload", choices=["c4", "c3", "c5", "c2", "c1", "qstep", "variance"], default="c4")
     ap.add_argument("--bucket", type=int, default=0, help="override the bucket size (c5 sweep)")
     ap.add_argument("--d", type=int, default=0, help="vector length for --workload c2")
     ap.add_argument("--scale-mode", choices=["norm", "max", "fixed"], default="norm",
                     help="bucket scale of --workload c2")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the short runs of C1, C2, C3, C5")
+    ap.add_argument("--no-sustained", action="store_true")
+    ap.add_argument("--sustained-seconds", type=float, default=0.8)
     ap.add_argument("--cpu-sample-elems", type=int, default=25_557_032)
     ap.add_argument("--ref-sample-elems", type=int, default=4_194_304)
-    args = ap.parse_args()
+    args = ap.parse_args(argv)
+    if args.gpus < 1:
+        raise SystemExit("bench.py: --gpus must be at least 1")
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
+    launched = "WORLD_SIZE" in os.environ
+    if launched and int(os.environ["WORLD_SIZE"]) != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but WORLD_SIZE={os.environ['WORLD_SIZE']}: start "
+                         f"one rank per GPU (torchrun --nproc-per-node {args.gpus}) or drop the variable")
     if args.impl == "reference":
         run_reference(args)
-    else:
-        run_ours(args)
+        return 0
+    if args.gpus > 1 and not launched:
+        # started plainly with --gpus N: become N ranks, one replica per GPU
+        import torch
+        have = torch.cuda.device_count()
+        if have < args.gpus:
+            raise SystemExit(f"bench.py: --gpus {args.gpus} but {have} CUDA device(s) visible")
+        return subprocess.call(torchrun_command(args.gpus, argv))
+    run_ours(args)
+    return 0
 
 
 if __name__ == "__main__":
-    main()
+    sys.exit(main())

@@ -542,6 +542,43 @@ def test_lr_gradient_matches_oracle_and_quantised_gradient_step(m, d):
 
 
 # ------------------------------------------------------ argument checking ----
+def test_quantisation_noise_of_gradient_and_epoch_delta_match_lemma_1():
+    """Gradient compression (QSGD baseline of Sec. 5, delta = ||g|| per bucket) against compression
+    of the epoch delta (Sec. 2.2) on a logistic problem, same width and bucket: for both vectors
+    the library's E||Q(v) - v||^2 over many draws equals Lemma 1's closed form
+    sum delta^2 p (1 - p) -- computed here by the CPU oracle's scales and exact fractions -- and
+    stays below d * delta^2 / 4; one draw of each is bit-identical to the oracle's."""
+    import bench
+    n_local, d, batch, lr, bucket = 256, 8192, 32, 0.1, 512
+    X, y, _ = synthetic.logistic_problem(n_local, d, seed=77)
+    c = G.ctx()
+    tX, ty = G.dev(X), G.dev(y)
+    w = torch.zeros(d, dtype=torch.float32, device="cuda")
+    g = torch.empty(d, dtype=torch.float32, device="cuda")
+    u = torch.zeros((1, d), dtype=torch.float32, device="cuda")
+    c.qesgd_lr_gradient(tX[:batch].contiguous(), ty[:batch].contiguous(), batch, d, w, g)
+    c.qesgd_lr_local_epoch_batch(tX, ty, n_local, d, 1, batch, lr, u, d)
+    torch.cuda.synchronize()
+    z = (u[0] - w).contiguous()
+    for bits, s in ((8, 127), (2, 1)):
+        for name, v in (("gradient", g), ("epoch delta", z)):
+            got = bench.quantisation_variance(c, v, bucket, s, bits, draws=64)
+            hv = v.cpu().numpy()
+            # closed form from the oracle's side: its scales, exact fractional parts
+            _, r_scales, _ = ref.encode(hv, None, bucket, s, bits, ref.SCALE_NORM, 5, 0, 0)
+            delta = np.repeat((r_scales / np.float32(s)).astype(np.float64), bucket)[:d]
+            r = np.abs(hv.astype(np.float64)) / delta
+            p = r - np.floor(r)
+            closed = float((delta ** 2 * p * (1 - p)).sum())
+            assert abs(got["closed_form"] - closed) <= 1e-9 * closed, name
+            # 64 draws x 8192 coordinates: the standard error of the mean is below 1 % even for 2-bit codes
+            assert abs(got["monte_carlo"] - closed) <= 0.04 * closed, (name, bits, got)
+            assert got["monte_carlo"] <= got["bound_d_delta2_over_4"]
+            gc, gs, _ = G.gpu_encode(hv, None, bucket, s, bits, ref.SCALE_NORM, 5, 0, 3)
+            wc, ws, _ = ref.encode(hv, None, bucket, s, bits, ref.SCALE_NORM, 5, 0, 3)
+            assert (gc == wc).all() and (gs.view(np.uint32) == ws.view(np.uint32)).all()
+
+
 def test_invalid_arguments_return_einval_and_launch_nothing():
     c = G.ctx()
     z = torch.zeros(4096, device="cuda")
