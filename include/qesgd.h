@@ -151,6 +151,24 @@ int qesgd_requantize(qesgd_ctx *ctx, float *u, const float *anchor, uint64_t d, 
                      uint32_t *codes_out, float *scales_out);
 
 /*
+ * The whole inner iteration of Algorithm 2 on logistic regression (its three lines: z^ = z -
+ * eta * grad f(u), z = Q(z^), u = w_t + z; Eq. 2 for the gradient step on the m rows of Xb):
+ * qesgd_lr_sgd_step followed by qesgd_requantize, without the updated parameter ever being
+ * written before it is quantised.  Two launches: the margin pass, then one kernel in which a
+ * CTA forms u^ = u - (lr/m) sum_j c_j x_j for a tile of 1024 columns in shared memory and
+ * requantises it there (u, zsum, codes_out, scales_out as for qesgd_requantize).  The update
+ * takes the arithmetic of qesgd_lr_sgd_step's two-pass form, so the result equals that call
+ * followed by qesgd_requantize bit for bit.  Shapes the fused kernel does not take (bucket
+ * above 1024, d not a multiple of 4, X or u not 16-byte aligned) run as those two calls.
+ * 1 <= m <= QESGD_MAX_LR_BATCH; other arguments as for qesgd_requantize.
+ */
+int qesgd_lr_qesgd_step(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32_t m, uint64_t d,
+                        float lr, float *u, const float *anchor, uint32_t bucket, uint32_t s,
+                        uint32_t bits, uint32_t scale_mode, float fixed_delta, uint64_t seed,
+                        uint32_t worker, uint32_t step, float *zsum, uint32_t *codes_out,
+                        float *scales_out);
+
+/*
  * Gradient compression on the push side (Sec. 3, remark after Algorithm 3; the QSGD
  * baseline of Sec. 5 quantises gradients with delta = ||g||): the K streams hold quantised
  * gradients, encoded with anchor == NULL, and the server takes

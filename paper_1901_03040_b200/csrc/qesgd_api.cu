@@ -211,6 +211,78 @@ int qesgd_requantize(qesgd_ctx *ctx, float *u, const float *anchor, uint64_t d, 
                        worker, step, codes_out, 0, scales_out, 0, u, zsum);
 }
 
+int qesgd_lr_qesgd_step(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32_t m, uint64_t d,
+                        float lr, float *u, const float *anchor, uint32_t bucket, uint32_t s,
+                        uint32_t bits, uint32_t scale_mode, float fixed_delta, uint64_t seed,
+                        uint32_t worker, uint32_t step, float *zsum, uint32_t *codes_out,
+                        float *scales_out)
+{
+    if (!ctx) return QESGD_EINVAL;
+    if (m < 1 || m > QESGD_MAX_LR_BATCH) return QESGD_EINVAL;
+    if (!valid_codec(bucket, s, bits) || scale_mode > QESGD_SCALE_FIXED) return QESGD_EINVAL;
+    if (scale_mode == QESGD_SCALE_FIXED && !(fixed_delta > 0.0f && fixed_delta <= 3.402823466e38f))
+        return QESGD_EINVAL;
+    if (d == 0) return QESGD_OK;
+    if (!Xb || !yb || !u || !anchor || !codes_out || !scales_out) return QESGD_EINVAL;
+    if (!aligned(Xb, 4) || !aligned(yb, 4) || !aligned(u, 4) || !aligned(anchor, 4)) return QESGD_EINVAL;
+    if (zsum && !aligned(zsum, 4)) return QESGD_EINVAL;
+    if (zsum && (aligned(u, 32) != aligned(zsum, 32))) return QESGD_EINVAL;
+    if (!aligned(codes_out, 16) || !aligned(scales_out, 16)) return QESGD_EINVAL;
+    const bool fused = bucket <= 1024u && d % 4 == 0 && aligned(Xb, 16) && aligned(u, 16) &&
+                       (uint64_t)m <= ctx->lr_work_floats;
+    if (!fused) {   // the same two steps as separate calls
+        const int rc = qesgd_lr_local_epoch_batch(ctx, Xb, yb, m, d, 1, m, lr, u, 0);
+        if (rc != QESGD_OK) return rc;
+        return qesgd_requantize(ctx, u, anchor, d, bucket, s, bits, scale_mode, fixed_delta, seed, worker,
+                                step, zsum, codes_out, scales_out);
+    }
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
+    QstepArgs q;
+    uint32_t parts = 0;
+    int e = qesgd_launch_lr_margins(Xb, yb, m, d, u, ctx->d_lr_work, ctx->lr_work_floats, ctx->stream, &parts);
+    if (e != 0) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    EncodeArgs &a = q.e;
+    const uint64_t nb = qesgd_num_buckets(d, bucket);
+    a.local = u;
+    a.local_stride = 0;
+    a.anchor = anchor;
+    a.d = d;
+    a.padded = nb * bucket;
+    a.log2_bucket = (uint32_t)log2_exact(bucket);
+    a.s = s;
+    a.fixed_scale = scale_mode == QESGD_SCALE_FIXED ? (float)s * fixed_delta : 0.0f;
+    for (uint32_t r = 0; r < 10; ++r) {
+        a.round_key[r][0] = (uint32_t)seed + r * 0x9E3779B9u;
+        a.round_key[r][1] = (uint32_t)(seed >> 32) + r * 0xBB67AE85u;
+    }
+    a.worker0 = worker;
+    a.epoch = step;
+    a.K = 1;
+    a.codes = codes_out;
+    a.code_stride = 0;
+    a.scales = scales_out;
+    a.scale_stride = 0;
+    a.status = ctx->d_status;
+    a.u_out = u;
+    a.zsum = zsum;
+    q.X = Xb;
+    q.y = yb;
+    q.m = m;
+    q.rate = lr / (float)m;
+    q.work = ctx->d_lr_work;
+    q.parts = parts;
+    switch (bits) {
+        case 2: e = qesgd_launch_lr_qstep_2(q, scale_mode, ctx->stream); break;
+        case 4: e = qesgd_launch_lr_qstep_4(q, scale_mode, ctx->stream); break;
+        default: e = qesgd_launch_lr_qstep_8(q, scale_mode, ctx->stream); break;
+    }
+    if (e != 0) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return QESGD_OK;
+}
+
 int qesgd_encode(qesgd_ctx *ctx, const float *local, const float *anchor, uint64_t d,
                  uint32_t bucket, uint32_t s, uint32_t bits, uint32_t scale_mode,
                  float fixed_delta, uint64_t seed, uint32_t worker, uint32_t epoch,

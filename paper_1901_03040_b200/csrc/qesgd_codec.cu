@@ -612,6 +612,91 @@ __global__ void __launch_bounds__(WARPS * 32, QESGD_ENCODE_MIN_WARPS / WARPS)
     encode_warp_tile<BITS, MODE, V, false, REQ>(a, z, warp_base, k, lane, warp, sh, 0u);
 }
 
+// ---------------------------------- update + requantise (Algorithm 2 inner step) ----
+// One inner iteration of QESGD on logistic regression after the margin pass: a CTA owns a
+// tile of 1024 columns, forms u^ = u - (lr/m) sum_j c_j x_j for them in shared memory (the
+// arithmetic of the plain update pass, in its order: rows split over four groups, group sums
+// added in group order), and its first warp then quantises u^ - w_t, writes u = w_t + Q(z^),
+// the running sum and the stream exactly as qesgd_requantize would.  The updated parameter
+// never travels to global memory before it is quantised.  Buckets of at most 1024 elements,
+// d a multiple of 4, 16-byte aligned X and u.
+constexpr int QS_COLS = 256;                   // columns per sub-tile: 64 groups of 4
+constexpr int QS_ROWGROUPS = 4;
+constexpr int QS_THREADS = (QS_COLS / 4) * QS_ROWGROUPS;
+constexpr int QS_TILE = 4 * CHUNK;             // columns per CTA
+
+template <int BITS, int MODE>
+__global__ void __launch_bounds__(QS_THREADS) qesgd_lr_qstep_kernel(const QstepArgs q)
+{
+    __shared__ float s_coef[QESGD_MAX_LR_BATCH];
+    __shared__ float4 s_sum[QS_ROWGROUPS][QS_COLS / 4];
+    __shared__ __align__(32) float s_u[QS_TILE];
+    __shared__ EncodeShared sh;
+    const EncodeArgs &a = q.e;
+    for (uint32_t j = threadIdx.x; j < q.m; j += blockDim.x) {
+        float margin = 0.0f;
+        for (uint32_t p = 0; p < q.parts; ++p) margin += q.work[(uint64_t)p * q.m + j];
+        const float yj = __ldg(q.y + j);
+        // -(lr/m) * c_j with c_j = -y_j / (1 + exp(y_j m_j))
+        s_coef[j] = q.rate * yj / (1.0f + expf(yj * margin));
+    }
+    __syncthreads();
+    const uint32_t cg = threadIdx.x % (QS_COLS / 4), rg = threadIdx.x / (QS_COLS / 4);
+    const uint64_t tile0 = (uint64_t)blockIdx.x * QS_TILE;
+#pragma unroll 1
+    for (int sub = 0; sub < QS_TILE / QS_COLS; ++sub) {
+        const uint64_t c = tile0 + (uint64_t)sub * QS_COLS + cg * 4u;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c + 4 <= a.d) {
+            const float *__restrict__ col = q.X + c;
+#pragma unroll 8
+            for (uint32_t j = rg; j < q.m; j += QS_ROWGROUPS) {
+                const float4 x = __ldg(reinterpret_cast<const float4 *>(col + (uint64_t)j * a.d));
+                const float cj = s_coef[j];
+                acc.x = fmaf(cj, x.x, acc.x);
+                acc.y = fmaf(cj, x.y, acc.y);
+                acc.z = fmaf(cj, x.z, acc.z);
+                acc.w = fmaf(cj, x.w, acc.w);
+            }
+        }
+        s_sum[rg][cg] = acc;
+        __syncthreads();
+        if (rg == 0) {
+            float4 uu = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c + 4 <= a.d) {
+                float4 t = s_sum[0][cg];
+#pragma unroll
+                for (int g = 1; g < QS_ROWGROUPS; ++g) {
+                    const float4 v = s_sum[g][cg];
+                    t.x = __fadd_rn(t.x, v.x); t.y = __fadd_rn(t.y, v.y);
+                    t.z = __fadd_rn(t.z, v.z); t.w = __fadd_rn(t.w, v.w);
+                }
+                uu = *reinterpret_cast<const float4 *>(a.local + c);
+                uu.x = __fadd_rn(uu.x, t.x); uu.y = __fadd_rn(uu.y, t.y);
+                uu.z = __fadd_rn(uu.z, t.z); uu.w = __fadd_rn(uu.w, t.w);
+            }
+            *reinterpret_cast<float4 *>(s_u + sub * QS_COLS + cg * 4u) = uu;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x >= 32) return;
+    // the first warp requantises the tile: z = u^ - w_t, zeros past d
+    const uint32_t lane = threadIdx.x;
+    float z[4][8];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        const uint64_t e0 = tile0 + (uint64_t)c * CHUNK + lane * 8u;
+        float w[8];
+        load_octet<false>(a.anchor, e0, a.d, w);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float uj = s_u[c * CHUNK + lane * 8u + j];
+            z[c][j] = (e0 + j < a.d) ? __fsub_rn(uj, w[j]) : 0.0f;
+        }
+    }
+    encode_warp_tile<BITS, MODE, 4, false, true>(a, z, tile0, 0u, lane, 0u, sh, 0u);
+}
+
 // ------------------------------------------------------------- decode -------
 // Signed value of slot j of a packed word: +-level * step.  The level is spliced
 // into the mantissa of 2^23 (exact integer -> float without the conversion pipe).
@@ -951,6 +1036,19 @@ int QESGD_CAT(qesgd_launch_encode_, QESGD_BITS)(const EncodeArgs &a, uint32_t K,
                                                 bool vec, int sm_count, cudaStream_t stream)
 {
     return (int)launch_encode_b<QESGD_BITS>(a, K, scale_mode, vec, sm_count, stream);
+}
+
+int QESGD_CAT(qesgd_launch_lr_qstep_, QESGD_BITS)(const QstepArgs &a, uint32_t scale_mode, cudaStream_t stream)
+{
+    const uint64_t tiles = (a.e.padded + QS_TILE - 1) / QS_TILE;
+    if (tiles == 0 || tiles > 0x7FFFFFFFull) return (int)cudaErrorInvalidValue;
+    dim3 grid((unsigned)tiles), block(QS_THREADS);
+    switch (scale_mode) {
+        case QESGD_SCALE_NORM: qesgd_lr_qstep_kernel<QESGD_BITS, 0><<<grid, block, 0, stream>>>(a); break;
+        case QESGD_SCALE_MAX: qesgd_lr_qstep_kernel<QESGD_BITS, 1><<<grid, block, 0, stream>>>(a); break;
+        default: qesgd_lr_qstep_kernel<QESGD_BITS, 2><<<grid, block, 0, stream>>>(a); break;
+    }
+    return (int)cudaGetLastError();
 }
 
 int QESGD_CAT(qesgd_launch_decode_, QESGD_BITS)(const DecodeArgs &a, bool vec, cudaStream_t stream)

@@ -46,6 +46,18 @@ struct EncodeArgs {
     float *zsum;            // per-step QESGD: running sum of Q(z), may be null
 };
 
+// One inner step of QESGD on logistic regression in two launches: the margin pass of the
+// plain step, then one kernel that forms the updated parameter of a tile in shared memory
+// and requantises it there.
+struct QstepArgs {
+    EncodeArgs e;           // the requantisation of u (K = 1, u_out = local = u)
+    const float *X, *y;     // the minibatch, m rows of d columns
+    uint32_t m;
+    float rate;             // lr / m
+    const float *work;      // partial margins of the margin pass: [parts][m]
+    uint32_t parts;
+};
+
 struct DecodeArgs {
     float *param;           // decode-average-apply: in/out; decode: out
     uint64_t d;
@@ -67,6 +79,9 @@ struct DecodeArgs {
                                 int sm_count, cudaStream_t stream);                             \
     int qesgd_launch_decode_##B(const DecodeArgs &a, bool vec, cudaStream_t stream);            \
     int qesgd_launch_decode_average_apply_##B(const DecodeArgs &a, bool vec, cudaStream_t stream);
+int qesgd_launch_lr_qstep_2(const QstepArgs &a, uint32_t scale_mode, cudaStream_t stream);
+int qesgd_launch_lr_qstep_4(const QstepArgs &a, uint32_t scale_mode, cudaStream_t stream);
+int qesgd_launch_lr_qstep_8(const QstepArgs &a, uint32_t scale_mode, cudaStream_t stream);
 QESGD_DECLARE_WIDTH(2)
 QESGD_DECLARE_WIDTH(4)
 QESGD_DECLARE_WIDTH(8)
@@ -103,6 +118,10 @@ int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float 
                          uint64_t y_worker_stride, uint32_t m, uint64_t d, uint32_t K, float lr,
                          float *u, uint64_t u_stride, float *work, uint64_t work_floats,
                          cudaStream_t stream, int *launched);
+// The margin pass alone (pass 1 of a step) for one worker; *parts_out receives the number of
+// partial margins per row that the pass leaves in `work` ([parts][m]).
+int qesgd_launch_lr_margins(const float *Xb, const float *yb, uint32_t m, uint64_t d, const float *u,
+                            float *work, uint64_t work_floats, cudaStream_t stream, uint32_t *parts_out);
 // Minibatch mean gradient at w into g (same two passes; the second writes instead of updating).
 int qesgd_launch_lr_gradient(const float *Xb, const float *yb, uint32_t m, uint64_t d,
                              const float *w, float *g, float *work, uint64_t work_floats,

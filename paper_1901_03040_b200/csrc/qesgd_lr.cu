@@ -234,6 +234,31 @@ int launch_lr_passes(const float *Xb, uint64_t x_worker_stride, const float *yb,
 
 }  // namespace
 
+int qesgd_launch_lr_margins(const float *Xb, const float *yb, uint32_t m, uint64_t d, const float *u,
+                            float *work, uint64_t work_floats, cudaStream_t stream, uint32_t *parts_out)
+{
+    LrArgs a;
+    a.X = Xb; a.x_stride = 0;
+    a.y = yb; a.y_stride = 0;
+    a.m = m; a.d = d;
+    a.rate = 0.0f;
+    a.u = u; a.dst = nullptr; a.accumulate = 0u; a.u_stride = 0;
+    a.work = work;
+    const uint64_t nseg = (d + SEG - 1) / SEG;
+    uint64_t parts = work_floats / (uint64_t)m;
+    if (parts > (uint64_t)MAX_PARTS) parts = MAX_PARTS;
+    if (parts > nseg) parts = nseg;
+    if (parts == 0 || nseg > 0xFFFFFFFFull) return (int)cudaErrorInvalidValue;
+    a.parts = (uint32_t)parts;
+    a.nseg = (uint32_t)nseg;
+    const bool vec = (d % 4 == 0) && (((uintptr_t)Xb | (uintptr_t)u) % 16 == 0);
+    dim3 g1((unsigned)parts, 1), b1(256);
+    if (vec) qesgd_lr_margin_kernel<true><<<g1, b1, 0, stream>>>(a);
+    else qesgd_lr_margin_kernel<false><<<g1, b1, 0, stream>>>(a);
+    *parts_out = a.parts;
+    return (int)cudaGetLastError();
+}
+
 int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float *yb,
                          uint64_t y_worker_stride, uint32_t m, uint64_t d, uint32_t K, float lr,
                          float *u, uint64_t u_stride, float *work, uint64_t work_floats,

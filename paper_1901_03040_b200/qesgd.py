@@ -40,6 +40,8 @@ SIGNATURES = {
                                   _u64, _u32, _u32, _vp, _u64, _vp, _u64]),
     "qesgd_requantize": (_int, [_vp, _vp, _vp, _u64, _u32, _u32, _u32, _u32, _f32, _u64, _u32, _u32,
                                 _vp, _vp, _vp]),
+    "qesgd_lr_qesgd_step": (_int, [_vp, _vp, _vp, _u32, _u64, _f32, _vp, _vp, _u32, _u32, _u32, _u32, _f32,
+                                   _u64, _u32, _u32, _vp, _vp, _vp]),
     "qesgd_decode_average_apply": (_int, [_vp, _vp, _u64, _u32, _vp, _u64, _vp, _u64, _u32, _u32,
                                           _u32]),
     "qesgd_decode_average_axpy": (_int, [_vp, _vp, _u64, _u32, _vp, _u64, _vp, _u64, _u32, _u32,
@@ -141,6 +143,12 @@ class Context:
         self._check(lib.qesgd_requantize(self._h, _ptr(u), _ptr(anchor), d, bucket, s, bits,
                                          scale_mode, fixed_delta, seed, worker, step, _ptr(zsum),
                                          _ptr(codes_out), _ptr(scales_out)))
+
+    def qesgd_lr_qesgd_step(self, Xb, yb, m, d, lr, u, anchor, bucket, s, bits, scale_mode, seed, worker,
+                            step, zsum, codes_out, scales_out, fixed_delta=0.0):
+        self._check(lib.qesgd_lr_qesgd_step(self._h, _ptr(Xb), _ptr(yb), m, d, lr, _ptr(u), _ptr(anchor),
+                                            bucket, s, bits, scale_mode, fixed_delta, seed, worker, step,
+                                            _ptr(zsum), _ptr(codes_out), _ptr(scales_out)))
 
     # -- server side ---------------------------------------------------------
     def qesgd_decode_average_apply(self, param, d, K, codes, code_stride, scales, scale_stride,

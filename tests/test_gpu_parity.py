@@ -498,6 +498,59 @@ def test_qesgd_inner_loop_on_the_gpu_follows_the_oracle():
 
 
 # ------------------------------------------- gradient compression (push side) ---
+@pytest.mark.parametrize("m,d,bucket,bits,s,mode,fused", [
+    (64, 65536, 512, 8, 127, ref.SCALE_NORM, True),    # the benchmark's logistic shape
+    (33, 4100, 64, 4, 7, ref.SCALE_MAX, True),         # ragged last tile, odd row count
+    (256, 8192, 1024, 2, 1, ref.SCALE_FIXED, True),    # widest bucket the fused kernel takes
+    (64, 8192, 4096, 8, 100, ref.SCALE_NORM, False),   # bucket above 1024: the two calls
+    (20, 1002, 128, 4, 7, ref.SCALE_NORM, False),      # d not a multiple of 4: the two calls
+])
+def test_fused_inner_step_equals_step_then_requantize(m, d, bucket, bits, s, mode, fused):
+    """Algorithm 2's inner iteration as one call: gradient step (Eq. 2) on the minibatch, then
+    z = Q(z^), u = w_t + z and the running sum.  The gradient step is tolerance-equal to the
+    fp64 oracle; from the GPU's own updated parameter on (hand-off) everything must equal the
+    oracle's requantisation bit for bit: u, running sum, codes, scales."""
+    X, y, _ = synthetic.logistic_problem(m, d, seed=m + d)
+    w = synthetic.anchor_vector(d, seed=8)
+    u0 = (w + _delta(d, 9, sigma=2e-3)).astype(np.float32)
+    zsum0 = _delta(d, 10, sigma=1e-3)
+    lr, fixed = 0.3, 4e-3 / s
+    c = G.ctx()
+    tX, ty = G.dev(X), G.dev(y)
+    # the gradient step alone, in the arithmetic the fused call uses
+    u1 = G.dev(u0)
+    if fused:
+        qesgd.qesgd_lr_sgd_step_noalloc(None, tX, ty, m, d, lr, u1)      # always the two-pass form
+    else:
+        c.qesgd_lr_sgd_step(tX, ty, m, d, lr, u1)
+    torch.cuda.synchronize()
+    u1 = u1.cpu().numpy()
+    _lr_close(u1, ref.lr_sgd_step(X, y, lr, u0))
+    want_u, want_zsum, want_codes, want_scales, want_st = ref.requantize(
+        u1, w, bucket, s, bits, mode, 21, 3, 7, zsum=zsum0, fixed_delta=fixed)
+    # the fused call from the same start
+    nb, cb = qesgd.num_buckets(d, bucket), qesgd.code_bytes(d, bucket, bits)
+    tu = torch.full((d + 8,), 55.0, dtype=torch.float32, device="cuda")
+    tu[:d] = G.dev(u0)
+    tz = torch.full((d + 8,), 66.0, dtype=torch.float32, device="cuda")
+    tz[:d] = G.dev(zsum0)
+    codes = torch.full((cb + 64,), 0xAB, dtype=torch.uint8, device="cuda")
+    scales = torch.full((nb + 16,), -7.0, dtype=torch.float32, device="cuda")
+    launches = c.qesgd_launch_count()
+    c.qesgd_lr_qesgd_step(tX, ty, m, d, lr, tu[:d], G.dev(w), bucket, s, bits, mode, 21, 3, 7, tz[:d],
+                          codes, scales, fixed_delta=fixed)
+    assert c.qesgd_status() == want_st
+    if fused:
+        assert c.qesgd_launch_count() - launches == 2      # margin pass + the fused kernel
+    assert (tu[d:] == 55.0).all().item() and (tz[d:] == 66.0).all().item()
+    assert (codes[cb:] == 0xAB).all().item() and (scales[nb:] == -7.0).all().item()
+    got_u, got_zsum = tu[:d].cpu().numpy(), tz[:d].cpu().numpy()
+    assert (scales[:nb].cpu().numpy().view(np.uint32) == want_scales.view(np.uint32)).all()
+    assert (codes[:cb].cpu().numpy().view(np.uint32) == want_codes).all()
+    assert (got_u.view(np.uint32) == want_u.view(np.uint32)).all()
+    assert (got_zsum.view(np.uint32) == want_zsum.view(np.uint32)).all()
+
+
 @pytest.mark.parametrize("alpha", [-0.1, 1.0, -3.5])
 @pytest.mark.parametrize("K,bucket,bits,s", [(4, 128, 4, 7), (16, 256, 2, 1), (3, 1024, 8, 127)])
 def test_decode_average_axpy_matches_oracle(K, bucket, bits, s, alpha):
@@ -570,7 +623,7 @@ def test_quantisation_noise_of_gradient_and_epoch_delta_match_lemma_1():
             r = np.abs(hv.astype(np.float64)) / delta
             p = r - np.floor(r)
             closed = float((delta ** 2 * p * (1 - p)).sum())
-            assert abs(got["closed_form"] - closed) <= 1e-9 * closed, name
+            assert abs(got["closed_form"] - closed) <= 1e-6 * closed, name
             # 64 draws x 8192 coordinates: the standard error of the mean is below 1 % even for 2-bit codes
             assert abs(got["monte_carlo"] - closed) <= 0.04 * closed, (name, bits, got)
             assert got["monte_carlo"] <= got["bound_d_delta2_over_4"]
