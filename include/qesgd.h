@@ -62,6 +62,8 @@ extern "C" {
 
 #define QESGD_STATUS_NONFINITE 1u /* a bucket held NaN/Inf or its norm overflowed fp32 */
 #define QESGD_STATUS_TIMEOUT 2u   /* a bounded wait inside the local-epoch kernel ran out   */
+#define QESGD_STATUS_RANGE 4u     /* debug build only: a codec kernel computed an index outside
+                                     its buffer; the access was skipped                       */
 
 #define QESGD_MAX_WORKERS 64u
 #define QESGD_MIN_BUCKET 64u
@@ -273,6 +275,14 @@ int qesgd_lr_sgd_step_noalloc(void *cuda_stream, const float *Xb, const float *y
 
 /* Waits for the stream, copies the status word to *flags_out (host) and clears it. */
 int qesgd_status(qesgd_ctx *ctx, uint32_t *flags_out);
+/* 1 if the library was built with QESGD_DEBUG (the codec kernels then check every store index,
+ * and the indices of their code and scale loads, against the extent of the buffer, skip an
+ * access that falls outside and set QESGD_STATUS_RANGE instead of faulting), else 0. */
+int qesgd_debug_build(void);
+/* Debug build only: runs the range check on an index that is out of range by construction (no
+ * memory access is made), so that QESGD_STATUS_RANGE appears in the status word; in a release
+ * build it returns QESGD_EINVAL and enqueues nothing. */
+int qesgd_debug_range_selftest(qesgd_ctx *ctx);
 /* Number of kernels this context has launched since creation. */
 uint64_t qesgd_launch_count(const qesgd_ctx *ctx);
 /* Last cudaError_t seen by this context (0 if none). */

@@ -12,6 +12,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libqesgd.so")
+LIB_DEBUG = os.path.join(HERE, "libqesgd_debug.so")
 
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 COMMON = ["-O3", "-std=c++17", "-lineinfo", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"),
@@ -41,15 +42,20 @@ def _stale(target, sources):
     return any(os.path.getmtime(s) > t for s in sources)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """Builds libqesgd.so, or with debug=True libqesgd_debug.so: the same library compiled with
+    -DQESGD_DEBUG (the codec kernels check their indices and set QESGD_STATUS_RANGE)."""
     os.makedirs(OBJ, exist_ok=True)
     headers = [os.path.join(CSRC, "qesgd_internal.h"), os.path.join(ROOT, "include", "qesgd.h"),
                os.path.abspath(__file__)]
     nvcc = _nvcc()
     objs = []
     procs = []
+    lib = LIB_DEBUG if debug else LIB
     for name, objname, extra in UNITS:
         src = os.path.join(CSRC, name)
+        if debug:
+            objname, extra = "debug_" + objname, extra + ["-DQESGD_DEBUG"]
         obj = os.path.join(OBJ, objname)
         objs.append(obj)
         if force or _stale(obj, [src] + headers):
@@ -61,11 +67,11 @@ def build(force: bool = False, verbose: bool = False) -> str:
             sys.stderr.write(out)
         if p.returncode != 0:
             raise RuntimeError("nvcc failed: " + " ".join(cmd))
-    if force or procs or _stale(LIB, objs):
-        cmd = [nvcc] + ARCH + ["-shared", "-o", LIB] + objs
+    if force or procs or _stale(lib, objs):
+        cmd = [nvcc] + ARCH + ["-shared", "-o", lib] + objs
         subprocess.run(cmd, check=True)
-    return LIB
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -321,6 +321,7 @@ int qesgd_decode_average_axpy(qesgd_ctx *ctx, float *param, uint64_t d, uint32_t
     a.code_stride = K > 1 ? code_stride : 0;
     a.scales = scales;
     a.scale_stride = K > 1 ? scale_stride : 0;
+    a.status = ctx->d_status;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
     const int e = qesgd_launch_decode_average_apply(a, bits, aligned(param, 32), ctx->stream);
@@ -357,6 +358,7 @@ int qesgd_decode(qesgd_ctx *ctx, const uint32_t *codes, const float *scales, uin
     a.code_stride = 0;
     a.scales = scales;
     a.scale_stride = 0;
+    a.status = ctx->d_status;
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
     const int e = qesgd_launch_decode(a, bits, aligned(out, 32), ctx->stream);
@@ -444,6 +446,30 @@ int qesgd_status(qesgd_ctx *ctx, uint32_t *flags_out)
     if (e == cudaSuccess) e = cudaStreamSynchronize(ctx->stream);
     if (e != cudaSuccess) return cuda_fail(ctx, (int)e);
     return QESGD_OK;
+}
+
+int qesgd_debug_build(void)
+{
+#ifdef QESGD_DEBUG
+    return 1;
+#else
+    return 0;
+#endif
+}
+
+int qesgd_debug_range_selftest(qesgd_ctx *ctx)
+{
+    if (!ctx) return QESGD_EINVAL;
+#ifdef QESGD_DEBUG
+    DeviceGuard guard(ctx->device);
+    if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
+    const int e = qesgd_launch_range_selftest(ctx->d_status, ctx->stream);
+    if (e != 0) return cuda_fail(ctx, e);
+    ctx->launches += 1;
+    return QESGD_OK;
+#else
+    return QESGD_EINVAL;
+#endif
 }
 
 uint64_t qesgd_launch_count(const qesgd_ctx *ctx) { return ctx ? ctx->launches : 0; }

@@ -475,8 +475,10 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
         }
         if (inside) {      // the first lane of every bucket writes its scale
             if (!wide) {
-                if ((off & bucket_mask) == 0u) sbase[off >> lb] = scale;
-            } else if (off == 0u && wide_first) {
+                if ((off & bucket_mask) == 0u &&
+                    QESGD_IN_RANGE(a.status, ((warp_base + off) >> lb) < (a.padded >> lb)))
+                    sbase[off >> lb] = scale;
+            } else if (off == 0u && wide_first && QESGD_IN_RANGE(a.status, (warp_base >> lb) < (a.padded >> lb))) {
                 sbase[0] = scale;
             }
         }
@@ -520,7 +522,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
                 w[j] = __fadd_rn(w[j], v[j]);
             }
             if (FULL) {
-                st256(a.u_out + go, w);
+                if (QESGD_IN_RANGE(a.status, e0 + 8 <= a.d)) st256(a.u_out + go, w);
             } else {
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
@@ -533,7 +535,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
 #pragma unroll
                 for (int j = 0; j < 8; ++j) zs[j] = __fadd_rn(zs[j], v[j]);
                 if (FULL) {
-                    st256(a.zsum + go, zs);
+                    if (QESGD_IN_RANGE(a.status, e0 + 8 <= a.d)) st256(a.zsum + go, zs);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 8; ++j)
@@ -543,7 +545,7 @@ __device__ __forceinline__ void encode_warp_tile(const EncodeArgs &a, float (&z)
         }
         uint32_t out[2];
         pack_octet<BITS>(X, Z, out);
-        if (inside) {
+        if (inside && QESGD_IN_RANGE(a.status, warp_base + off + 8 <= a.padded)) {
             uint8_t *const q = cbase + c * (CHUNK * BITS / 8);
             if (BITS == 8) {
                 *reinterpret_cast<uint2 *>(q) = make_uint2(out[0], out[1]);
@@ -734,9 +736,13 @@ __global__ void __launch_bounds__(256) qesgd_decode_kernel(const DecodeArgs a)
     const uint64_t eb = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8u;
     if (eb >= a.d) return;
     const uint8_t *__restrict__ codes = reinterpret_cast<const uint8_t *>(a.codes);
-    uint32_t w[2];
-    load_codes<BITS>(codes, eb, w);
-    const float step = __fdiv_rn(__ldg(a.scales + (eb >> a.log2_bucket)), (float)a.s);
+    uint32_t w[2] = {0u, 0u};
+    float sc = 0.0f;
+    if (QESGD_IN_RANGE(a.status, eb + 8 <= (a.nb << a.log2_bucket))) {
+        load_codes<BITS>(codes, eb, w);
+        sc = __ldg(a.scales + (eb >> a.log2_bucket));
+    }
+    const float step = __fdiv_rn(sc, (float)a.s);
     float v[8];
     constexpr int PER_WORD = 32 / BITS;
 #pragma unroll
@@ -848,6 +854,9 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
         // is a multiple of 64, so a lane's 8, 16 or 32 elements are inside it or outside it.
         const uint64_t safe_eb = eb[c] < (a.nb << lb) ? eb[c] : warp_eb;
         cp[c] = reinterpret_cast<const uint8_t *>(a.codes) + (safe_eb >> 3) * (uint64_t)BITS;
+#ifdef QESGD_DEBUG
+        if (!QESGD_IN_RANGE(a.status, safe_eb + LANE_ELEMS <= (a.nb << lb))) cp[c] = reinterpret_cast<const uint8_t *>(a.codes);
+#endif
 #pragma unroll
         for (int o = 0; o < OPL; ++o)
 #pragma unroll
@@ -882,7 +891,9 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
     auto fetch_scale = [&](uint32_t kfirst) {
         const uint32_t kk = kfirst + lane / nbw;
         const uint64_t bb = bucket0 + (lane % nbw);
-        return (kk < a.K && bb < a.nb) ? __ldg(a.scales + (uint64_t)kk * a.scale_stride + bb) : 0.0f;
+        return (kk < a.K && bb < a.nb && QESGD_IN_RANGE(a.status, bb < a.nb))
+                   ? __ldg(a.scales + (uint64_t)kk * a.scale_stride + bb)
+                   : 0.0f;
     };
     uint32_t cw[BATCH][W][2], nx[BATCH][W][2];
     fetch(0u, cw);
@@ -959,7 +970,7 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
             }
             const uint64_t e0 = eb[c] + 8u * o;
             if (VEC && e0 + 8 <= a.d) {
-                st256(a.param + e0, w[o]);
+                if (QESGD_IN_RANGE(a.status, e0 + 8 <= a.d)) st256(a.param + e0, w[o]);
             } else {
 #pragma unroll
                 for (int j = 0; j < 8; ++j)
@@ -1022,7 +1033,22 @@ cudaError_t launch_encode_b(const EncodeArgs &a, uint32_t K, uint32_t mode, bool
     }
 }
 
+#if defined(QESGD_DEBUG) && QESGD_BITS == 2
+__global__ void qesgd_range_selftest_kernel(uint32_t *status, uint64_t index, uint64_t limit)
+{
+    if (QESGD_IN_RANGE(status, index < limit)) status[1] = 1u;   // never: the index is outside
+}
+#endif
+
 }  // namespace
+
+#if defined(QESGD_DEBUG) && QESGD_BITS == 2
+int qesgd_launch_range_selftest(uint32_t *status, cudaStream_t stream)
+{
+    qesgd_range_selftest_kernel<<<1, 1, 0, stream>>>(status, 7u, 7u);
+    return (int)cudaGetLastError();
+}
+#endif
 
 // This file is compiled once per code width (-DQESGD_BITS=2, 4, 8) so that the three sets
 // of kernel instantiations build in parallel; qesgd_api.cu picks the set at run time.

@@ -7,6 +7,14 @@
 
 #include "qesgd.h"
 
+// Debug build: an index is checked against its limit; outside it the status word receives
+// QESGD_STATUS_RANGE and the caller skips the access.  Release build: always true, no code.
+#ifdef QESGD_DEBUG
+#define QESGD_IN_RANGE(status, cond) ((cond) ? true : (atomicOr((status), QESGD_STATUS_RANGE), false))
+#else
+#define QESGD_IN_RANGE(status, cond) true
+#endif
+
 struct qesgd_ctx {
     int device;
     cudaStream_t stream;
@@ -70,7 +78,9 @@ struct DecodeArgs {
     uint64_t code_stride;   // bytes
     const float *scales;
     uint64_t scale_stride;  // elements
+    uint32_t *status;
 };
+int qesgd_launch_range_selftest(uint32_t *status, cudaStream_t stream);
 
 // Launchers.  Return a cudaError_t as int.  qesgd_codec.cu is compiled once per code width
 // and defines the *_2, *_4, *_8 functions; the width-dispatching wrappers are inline here.

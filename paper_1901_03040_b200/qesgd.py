@@ -8,11 +8,14 @@ import ctypes as C
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libqesgd.so")
+# QESGD_DEBUG=1 in the environment selects the debug build of the same library (index checks in
+# the codec kernels, QESGD_STATUS_RANGE); build it with `python -m paper_1901_03040_b200.build --debug`
+LIB_PATH = os.path.join(_HERE, "libqesgd_debug.so" if os.environ.get("QESGD_DEBUG") == "1" else "libqesgd.so")
 
 SCALE_NORM, SCALE_MAX, SCALE_FIXED = 0, 1, 2
 STATUS_NONFINITE = 1
 STATUS_TIMEOUT = 2
+STATUS_RANGE = 4
 OK, EINVAL, ECUDA, ENOMEM, ELIMIT = 0, -1, -2, -3, -4
 MAX_WORKERS, MIN_BUCKET, MAX_BUCKET, MAX_LR_BATCH = 64, 64, 8192, 1024
 NOALLOC_MAX_LR_BATCH = 256
@@ -53,6 +56,8 @@ SIGNATURES = {
     "qesgd_lr_local_epoch_batch": (_int, [_vp, _vp, _vp, _u64, _u64, _u32, _u32, _f32, _vp, _u64]),
     "qesgd_lr_sgd_step_noalloc": (_int, [_vp, _vp, _vp, _u32, _u64, _f32, _vp]),
     "qesgd_status": (_int, [_vp, C.POINTER(_u32)]),
+    "qesgd_debug_build": (_int, []),
+    "qesgd_debug_range_selftest": (_int, [_vp]),
     "qesgd_launch_count": (_u64, [_vp]),
     "qesgd_last_cuda_error": (_int, [_vp]),
     "qesgd_strerror": (C.c_char_p, [_int]),
