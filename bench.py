@@ -870,7 +870,7 @@ def run_c1(args, device, world, rank):
         e[3].record(stream)
         torch.cuda.synchronize()
         losses.append(loss(param))
-        if it == 0:   # round 1 (from w = 0), outside every timed region
+        if it == 0:   # the first QESGD round (from w = 0), outside every timed region
             first_round = c1_first_round(args, rank, world, X, y, u, codes, scales, param, loss,
                                          (n_local, d, K, batch, lr, B, s, bits))
         if it >= args.warmup:
@@ -903,7 +903,7 @@ def run_c1(args, device, world, rank):
         o = first_round["oracle"]
         line["cpu_baseline"] = {"value": 1e3 * (o["oracle_local_epoch_s"] + o["oracle_codec_s"]), "unit": "ms",
                                 "cores": 1, "kind": "oracle",
-                                "sample": "the whole of round 1: four local epochs, encode of the four "
+                                "sample": "the whole of the first QESGD round: four local epochs, encode of the four "
                                           "workers, decode-average-apply"}
     ctx.close()
     return line
@@ -992,7 +992,7 @@ def run_variance(args, device, world, rank):
 
 
 def c1_first_round(args, rank, world, X, y, u, codes, scales, param, loss, shape):
-    """Round 1 of C1 looked at from outside the timed region: the loss the unquantised average of
+    """The first QESGD round of C1 looked at from outside the timed region: the loss the unquantised average of
     the workers' parameters would have given (Sec. 5 claims 8 bits lose nothing against plain
     SGD), and, with the CPU oracle, the same round on the host: the oracle's local epochs against
     the GPU's (tolerance), then hand-off parity -- the oracle encodes the GPU's u_k and its codes
