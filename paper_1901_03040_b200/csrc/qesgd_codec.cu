@@ -820,10 +820,16 @@ __device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], int o,
 // needs are computed once per warp (one division per lane) and handed out by shuffle;
 // code words are fetched several workers at a time so that independent loads are in
 // flight before the first is used.
-template <int BITS, bool VEC, int W>
+// KS > 0: the number of workers is that compile-time constant and the worker loop is unrolled
+// completely (no loop counter, no predicates on the worker index).  Measured: 14 % faster for
+// 8-bit and 4 % for 4-bit codes at K = 8, but 9 % slower for 2-bit codes at K = 16, whose
+// unrolled loop (16 workers x 32 codes per lane) no longer fits the instruction cache; the
+// launcher therefore uses it for 4- and 8-bit codes only.
+template <int BITS, bool VEC, int W, int KS = 0>
 __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
     qesgd_decode_average_apply_kernel(const DecodeArgs a)
 {
+    const uint32_t K = KS ? (uint32_t)KS : a.K;
     constexpr int OPL = 8 / BITS;                 // octets per lane and chunk: 4, 2, 1
     constexpr int LANE_ELEMS = 8 * OPL;
     constexpr uint32_t WCHUNK = 32 * LANE_ELEMS;  // elements per chunk: 1024, 512, 256
@@ -877,7 +883,7 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
 #pragma unroll
             for (int c = 0; c < W; ++c) {
                 dst[i][c][0] = dst[i][c][1] = 0u;
-                if (kfirst + i < a.K) {
+                if (kfirst + i < K) {
                     const uint2 v = __ldg(reinterpret_cast<const uint2 *>(
                         cp[c] + (uint64_t)(kfirst + i) * a.code_stride));
                     dst[i][c][0] = v.x;
@@ -891,7 +897,7 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
     auto fetch_scale = [&](uint32_t kfirst) {
         const uint32_t kk = kfirst + lane / nbw;
         const uint64_t bb = bucket0 + (lane % nbw);
-        return (kk < a.K && bb < a.nb && QESGD_IN_RANGE(a.status, bb < a.nb))
+        return (kk < K && bb < a.nb && QESGD_IN_RANGE(a.status, bb < a.nb))
                    ? __ldg(a.scales + (uint64_t)kk * a.scale_stride + bb)
                    : 0.0f;
     };
@@ -899,19 +905,22 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
     fetch(0u, cw);
     float sc_next = fetch_scale(0u);
     float st = 0.0f;
-    for (uint32_t kb = 0; kb < a.K; kb += BATCH) {
+#pragma unroll
+    for (uint32_t kb = 0; kb < (KS ? (uint32_t)KS : a.K); kb += BATCH) {
         fetch(kb + BATCH, nx);
 #pragma unroll
         for (int i = 0; i < BATCH; ++i) {
             const uint32_t k = kb + i;
-            if (k < a.K) {   // uniform across the warp
-                if (k % per_pass == 0u) {   // a new pass: every lane computes one spacing
+            if (k < K) {   // uniform across the warp
+                // position of worker k inside its pass (per_pass is a power of two)
+                const uint32_t kp = KS ? (k & (per_pass - 1u)) : k % per_pass;
+                if (kp == 0u) {   // a new pass: every lane computes one spacing
                     st = __fdiv_rn(sc_next, sf);
                     sc_next = fetch_scale(k + per_pass);
                 }
 #pragma unroll
                 for (int c = 0; c < W; ++c) {
-                    const float step = __shfl_sync(FULL, st, (k % per_pass) * nbw + sub[c]);
+                    const float step = __shfl_sync(FULL, st, kp * nbw + sub[c]);
                     if (BITS == 4 && lut) {
                         // every lane holds the value of code (lane & 15) for this worker; a
                         // code is decoded by fetching its value from that lane of the same
@@ -1098,7 +1107,13 @@ int QESGD_CAT(qesgd_launch_decode_average_apply_, QESGD_BITS)(const DecodeArgs &
     const uint64_t blocks = (warps + wpc - 1) / wpc;
     if (blocks == 0 || blocks > 0x7FFFFFFFull) return (int)cudaErrorInvalidValue;
     dim3 grid((unsigned)blocks), block(QESGD_DAA_THREADS);
-    if (vec) qesgd_decode_average_apply_kernel<QESGD_BITS, true, W><<<grid, block, 0, stream>>>(a);
+    if (vec && QESGD_BITS != 2 && a.K == 8)
+        qesgd_decode_average_apply_kernel<QESGD_BITS, true, W, (QESGD_BITS != 2 ? 8 : 0)><<<grid, block, 0, stream>>>(a);
+    else if (vec && QESGD_BITS != 2 && a.K == 4)
+        qesgd_decode_average_apply_kernel<QESGD_BITS, true, W, (QESGD_BITS != 2 ? 4 : 0)><<<grid, block, 0, stream>>>(a);
+    else if (vec && QESGD_BITS == 8 && a.K == 16)
+        qesgd_decode_average_apply_kernel<QESGD_BITS, true, W, (QESGD_BITS == 8 ? 16 : 0)><<<grid, block, 0, stream>>>(a);
+    else if (vec) qesgd_decode_average_apply_kernel<QESGD_BITS, true, W><<<grid, block, 0, stream>>>(a);
     else qesgd_decode_average_apply_kernel<QESGD_BITS, false, W><<<grid, block, 0, stream>>>(a);
     return (int)cudaGetLastError();
 }
