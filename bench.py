@@ -155,7 +155,6 @@ def aggregate_over_ranks(ms_local, units_local, world, device=None, backend_read
 
 # --------------------------------------------------------------------- ours ---
 def make_round_inputs(w, device, seed=0):
-    import torch
     from paper_1901_03040_b200 import synthetic
     d, K = w["d"], w["K"]
     stride = (d + 7) // 8 * 8
@@ -328,7 +327,6 @@ def sustained_leg(rb, first_epoch, ms_per_step, peak, gpu_index, seconds=0.8):
 
 
 def run_ours(args):
-    import numpy as np
     import torch
     import torch.distributed as dist
 
@@ -831,7 +829,6 @@ def run_qstep(args, device, world, rank):
 def run_c1(args, device, world, rank):
     """End-to-end QESGD round on logistic regression: K=4 workers run one local epoch of
     minibatch-64 SGD from the anchor, encode (8-bit, bucket 512), server applies."""
-    import numpy as np
     import torch
     from paper_1901_03040_b200 import qesgd, synthetic
     n, d, K, batch, lr, B, s, bits = 8192, 65536, 4, 64, 0.1, 512, 127, 8
@@ -998,7 +995,6 @@ def c1_first_round(args, rank, world, X, y, u, codes, scales, param, loss, shape
     the GPU's (tolerance), then hand-off parity -- the oracle encodes the GPU's u_k and its codes
     and scales must equal the GPU's bit for bit, its applied parameter within 1e-6."""
     import numpy as np
-    import torch
     n_local, d, K, batch, lr, B, s, bits = shape
     out = {"loss_unquantised_average": loss(u.mean(0)), "loss_quantised": loss(param)}
     if not (rank == 0 and world == 1 and not args.no_cpu):
