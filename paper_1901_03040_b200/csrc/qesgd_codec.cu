@@ -825,8 +825,10 @@ __device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], int o,
 // 8-bit and 4 % for 4-bit codes at K = 8, but 9 % slower for 2-bit codes at K = 16, whose
 // unrolled loop (16 workers x 32 codes per lane) no longer fits the instruction cache; the
 // launcher therefore uses it for 4- and 8-bit codes only.
+// Register budget: 24 resident CTAs per SM, 28 for 4-bit codes (measured 4-5 % faster there,
+// slower for the other widths).
 template <int BITS, bool VEC, int W, int KS = 0>
-__global__ void __launch_bounds__(QESGD_DAA_THREADS, QESGD_DAA_MIN_CTAS)
+__global__ void __launch_bounds__(QESGD_DAA_THREADS, BITS == 4 ? QESGD_DAA_MIN_CTAS + 4 : QESGD_DAA_MIN_CTAS)
     qesgd_decode_average_apply_kernel(const DecodeArgs a)
 {
     const uint32_t K = KS ? (uint32_t)KS : a.K;
