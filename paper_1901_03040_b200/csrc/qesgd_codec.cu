@@ -745,8 +745,18 @@ __global__ void __launch_bounds__(256) qesgd_decode_kernel(const DecodeArgs a)
     const float step = __fdiv_rn(sc, (float)a.s);
     float v[8];
     constexpr int PER_WORD = 32 / BITS;
+    if (BITS == 2) {
+        // A two-bit code moved to bits 31 and 30 IS the float +-2.0 (level 1) or +-0.0 (level 0);
+        // times step/2 (exact: s = 1, so step is the scale, far above the subnormal range or 0)
+        // that is +-step or +-0 bit for bit, the value fl32(level * step) with the code's sign.
+        const float hs = __fmul_rn(step, 0.5f);
 #pragma unroll
-    for (int j = 0; j < 8; ++j) v[j] = code_value<BITS>(w[j / PER_WORD], j % PER_WORD, step);
+        for (int j = 0; j < 8; ++j)
+            v[j] = __fmul_rn(__uint_as_float((w[0] << (30 - 2 * j)) & 0xC0000000u), hs);
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = code_value<BITS>(w[j / PER_WORD], j % PER_WORD, step);
+    }
     if (VEC && eb + 8 <= a.d) {
         st256(a.param + eb, v);
     } else {
