@@ -125,10 +125,13 @@ int qesgd_encode_batch(qesgd_ctx *ctx, const float *local, uint64_t local_stride
  * Server side (last line of the server task of Algorithm 3, same average as the
  * last line of Algorithms 1 and 2):
  *   param_i <- param_i + (1/K) * sum_k (+-level_{k,i} * fl32(scale_{k,bucket(i)} / s))
- * param: float[d], updated in place, read once and written once.  Stream k starts
- * at codes + k*code_stride (BYTES) and scales + k*scale_stride (elements).
- * fp32 accumulation; result within 1e-6 * max(|param_i|, max_k scale) of the
- * exactly rounded value.  1 <= K <= 64.
+ * param: float[d], updated in place: every element receives exactly one add,
+ * fl32(param_i + fl32(sum_i * (1/K))), carried out by the memory system (a reduction,
+ * not a load and a store of the kernel), so the line is read and written once and the
+ * result does not depend on any order.  Stream k starts at codes + k*code_stride
+ * (BYTES) and scales + k*scale_stride (elements).  fp32 accumulation over k
+ * ascending; result within 1e-6 * max(|param_i|, max_k scale) of the exactly
+ * rounded value.  1 <= K <= 64.
  */
 int qesgd_decode_average_apply(qesgd_ctx *ctx, float *param, uint64_t d, uint32_t K,
                                const uint32_t *codes, uint64_t code_stride, const float *scales,

@@ -832,9 +832,9 @@ __device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], int o,
 // flight before the first is used.
 // KS > 0: the number of workers is that compile-time constant and the worker loop is unrolled
 // completely (no loop counter, no predicates on the worker index).  Measured: 14 % faster for
-// 8-bit and 4 % for 4-bit codes at K = 8, but 9 % slower for 2-bit codes at K = 16, whose
-// unrolled loop (16 workers x 32 codes per lane) no longer fits the instruction cache; the
-// launcher therefore uses it for 4- and 8-bit codes only.
+// 8-bit, 4 % for 4-bit and 4 % for 2-bit codes at K = 8, but slower for 2-bit codes at K = 4
+// (1 %) and at K = 16 (3-9 %: 16 workers x 32 codes per lane no longer fit the instruction
+// cache); the launcher picks accordingly.
 // Register budget: 24 resident CTAs per SM, 28 for 4-bit codes (measured 4-5 % faster there,
 // slower for the other widths).
 template <int BITS, bool VEC, int W, int KS = 0>
@@ -964,38 +964,53 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, BITS == 4 ? QESGD_DAA_MIN_C
                 cw[i][c][1] = nx[i][c][1];
             }
     }
-    // The parameter is fetched only now: its registers are not held through the worker loop
-    // (the other resident warps cover the latency), which lets more warps be resident.
+    // Apply: param += (alpha / K) * sum.  The warp never loads the parameter: every element
+    // gets exactly one add, done by the memory system (a vector reduction of four floats), so a
+    // warp's life ends with its last code word instead of a further round trip to memory, and the
+    // result, fl32(param + fl32(sum * alpha / K)), does not depend on any order.  A lane's
+    // elements are LANE_ELEMS consecutive floats, 32 to 128 bytes apart from the next lane's;
+    // the increments go through shared memory once so that every reduction instruction covers
+    // 512 consecutive bytes (32 lanes x 16 bytes).  Pieces of 16 bytes are stored at index
+    // P ^ ((P >> 3) & 7), which keeps both the lane-major writes and the piece-major reads free
+    // of bank conflicts for 2, 4 or 8 pieces per lane.
     const float inv_k = a.avg_scale;   // alpha / K
+    constexpr int NCH = LANE_ELEMS / 4;           // 16-byte pieces per lane and chunk: 8, 4, 2
+    __shared__ float4 s_inc[(QESGD_DAA_THREADS / 32) * W * 32 * NCH];
+    float4 *wt = s_inc + (threadIdx.x >> 5) * (W * 32 * NCH);
 #pragma unroll
     for (int c = 0; c < W; ++c) {
-        float w[OPL][8];
 #pragma unroll
         for (int o = 0; o < OPL; ++o) {
-            const uint64_t e0 = eb[c] + 8u * o;
-            if (VEC && e0 + 8 <= a.d) {
-                ld256_rw(a.param + e0, w[o]);
-            } else {
 #pragma unroll
-                for (int j = 0; j < 8; ++j) w[o][j] = (e0 + j < a.d) ? a.param[e0 + j] : 0.0f;
+            for (int h = 0; h < 2; ++h) {
+                float f0, f1, f2, f3;
+                unpack2(acc[c][o][2 * h], f0, f1);
+                unpack2(acc[c][o][2 * h + 1], f2, f3);
+                const uint32_t P = lane * NCH + 2 * o + h;
+                wt[c * 32 * NCH + (P ^ ((P >> 3) & 7u))] =
+                    make_float4(__fmul_rn(f0, inv_k), __fmul_rn(f1, inv_k), __fmul_rn(f2, inv_k),
+                                __fmul_rn(f3, inv_k));
             }
         }
+    }
+    __syncwarp();
 #pragma unroll
-        for (int o = 0; o < OPL; ++o) {
+    for (int c = 0; c < W; ++c) {
 #pragma unroll
-            for (int p = 0; p < 4; ++p) {
-                float lo, hi;
-                unpack2(acc[c][o][p], lo, hi);
-                w[o][2 * p] = __fmaf_rn(lo, inv_k, w[o][2 * p]);
-                w[o][2 * p + 1] = __fmaf_rn(hi, inv_k, w[o][2 * p + 1]);
-            }
-            const uint64_t e0 = eb[c] + 8u * o;
-            if (VEC && e0 + 8 <= a.d) {
-                if (QESGD_IN_RANGE(a.status, e0 + 8 <= a.d)) st256(a.param + e0, w[o]);
+        for (int i = 0; i < NCH; ++i) {
+            const uint32_t g = i * 32 + lane;     // piece g of the chunk: elements 4g .. 4g+3
+            const float4 v = wt[c * 32 * NCH + (g ^ ((g >> 3) & 7u))];
+            const uint64_t e = warp_eb + (uint64_t)c * WCHUNK + 4u * g;
+            float *q = a.param + e;
+            if (VEC && e + 4 <= a.d) {
+                if (QESGD_IN_RANGE(a.status, e + 4 <= a.d))
+                    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};"
+                                 :: "l"(q), "f"(v.x), "f"(v.y), "f"(v.z), "f"(v.w) : "memory");
             } else {
-#pragma unroll
-                for (int j = 0; j < 8; ++j)
-                    if (e0 + j < a.d) a.param[e0 + j] = w[o][j];
+                if (e < a.d) atomicAdd(q, v.x);
+                if (e + 1 < a.d) atomicAdd(q + 1, v.y);
+                if (e + 2 < a.d) atomicAdd(q + 2, v.z);
+                if (e + 3 < a.d) atomicAdd(q + 3, v.w);
             }
         }
     }
@@ -1119,8 +1134,8 @@ int QESGD_CAT(qesgd_launch_decode_average_apply_, QESGD_BITS)(const DecodeArgs &
     const uint64_t blocks = (warps + wpc - 1) / wpc;
     if (blocks == 0 || blocks > 0x7FFFFFFFull) return (int)cudaErrorInvalidValue;
     dim3 grid((unsigned)blocks), block(QESGD_DAA_THREADS);
-    if (vec && QESGD_BITS != 2 && a.K == 8)
-        qesgd_decode_average_apply_kernel<QESGD_BITS, true, W, (QESGD_BITS != 2 ? 8 : 0)><<<grid, block, 0, stream>>>(a);
+    if (vec && a.K == 8)
+        qesgd_decode_average_apply_kernel<QESGD_BITS, true, W, 8><<<grid, block, 0, stream>>>(a);
     else if (vec && QESGD_BITS != 2 && a.K == 4)
         qesgd_decode_average_apply_kernel<QESGD_BITS, true, W, (QESGD_BITS != 2 ? 4 : 0)><<<grid, block, 0, stream>>>(a);
     else if (vec && QESGD_BITS == 8 && a.K == 16)
