@@ -218,7 +218,12 @@ int qesgd_lr_local_epoch(qesgd_ctx *ctx, const float *X, const float *y, uint64_
  * of all K workers is ONE persistent kernel, launched cooperatively with one CTA per SM,
  * that stages every minibatch in shared memory by TMA and reads X from HBM once; its
  * CTAs exchange partial margins through the context's workspace, which the call clears
- * first.  Every wait the kernel loops on (for another CTA, another warp group, a copy) is
+ * first.  The partial margins of a row are summed across the CTAs as fixed-point integers
+ * (units of 2^-28 below 2^17 in magnitude, units of 2^-6 from there to 2^49), so the sum
+ * does not depend on the order in which the CTAs arrive; a NaN partial makes the row's
+ * margin NaN, an infinite one (or one of 2^49 or more, far beyond where the step
+ * coefficient saturates) makes it that infinity, and both then spread through u as they
+ * would in floating point.  Every wait the kernel loops on (for another CTA, another warp group, a copy) is
  * bounded by the context's wait limit (one second unless qesgd_set_wait_limit changed it):
  * should one run out, the kernel returns, u is left partly updated and
  * QESGD_STATUS_TIMEOUT is set in the status word; the context stays usable and the next call
@@ -228,7 +233,7 @@ int qesgd_lr_local_epoch(qesgd_ctx *ctx, const float *X, const float *y, uint64_
  * needs all its CTAs resident at once, so do not run it next to other kernels that occupy
  * the device for long.  Other shapes run one margin pass and one
  * update pass per minibatch, step t of every worker in the same launches.  Results are
- * deterministic (fixed summation order) on either path. */
+ * deterministic (order-free integer sums or a fixed summation order) on either path. */
 int qesgd_lr_local_epoch_batch(qesgd_ctx *ctx, const float *X, const float *y, uint64_t n_local,
                                uint64_t d, uint32_t K, uint32_t batch, float lr, float *u,
                                uint64_t u_stride);

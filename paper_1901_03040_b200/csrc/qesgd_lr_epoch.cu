@@ -13,11 +13,26 @@
 //                  cp.async.bulk.tensor global -> shared, completion on an mbarrier per
 //                  sub-tile); a producer warp issues the copies of tile i+2 as soon as the
 //                  consumer warps have released the buffer of tile i
-//   M(i)  margins of tile i over the CTA's columns -> partial[i % RING][row][cta],
-//         then fence + one atomic increment of counter[i]
-//   W(i)  wait until counter[i] == number of CTAs, sum the partials of every row in a
-//         fixed order, coefficients (lr/m) y_j / (1 + exp(y_j m_j)) into shared memory
+//   M(i)  margins of tile i over the CTA's columns; each row's partial margin is added, as a
+//         fixed-point integer, to the row's accumulator acc[i % RING][row] by one 64-bit
+//         reduction that also counts the contribution in the word's top bits
+//   W(i)  wait until every row's count equals the number of CTAs, margins from the sums,
+//         coefficients (lr/m) y_j / (1 + exp(y_j m_j)) into shared memory
 //   U(i)  u[cols] += sum_j coef_j x_j from the tile
+//
+// The exchange of the margins is what the epoch waits for, so it is one step: integer addition
+// is exact and commutes, so the sum over the CTAs needs no order, no second pass over 148
+// partials and -- the count travelling in the same word as the sum -- no fence between data and
+// signal; the result is the same in every run.  A word is count << 55 | sum, every contribution
+// adds 1 << 55 plus 2^45 + round(partial * 2^28) (the 2^45 keeps it positive; |partial| < 2^17;
+// up to 511 CTAs fit below the count).  A larger finite partial goes, in units of 2^-6 (the
+// spacing of fp32 at 2^17), into the second word of the row; a NaN is counted in the third word
+// and makes the margin NaN; an infinite partial, or one of 2^49 or more, is counted by sign in
+// the fourth and makes the margin that infinity (NaN if both signs occur), which the step
+// coefficient saturates on as it would on the number itself.  These rare kinds fence before they
+// count themselves in the first word.  The slot that tile i + RING/2 will use is cleared by one CTA
+// during M(i): every CTA has read it by then (it has taken part in tile i-2, hence finished
+// tile i-4) and none adds to it before it has seen that CTA's contributions to tile i+2.
 //
 // Where the minibatch has at most 64 rows the tile does not wait in shared memory between M
 // and U: right after M every thread moves its share of it into tensor memory (tcgen05.st;
@@ -26,8 +41,8 @@
 // one waits for the other CTAs; U reads the tile back with tcgen05.ld.  Larger minibatches
 // stay in shared memory and release their slots during U.
 //
-// Each tile's M, W, U is a chain of dependent round trips to global memory (fence, count,
-// partial margins) that lasts longer than the tile's own transfer from HBM.  The eight
+// Each tile's M, W, U is a chain of dependent round trips to global memory (reductions out,
+// sums back) that lasts longer than the tile's own transfer from HBM.  The eight
 // consumer warps therefore form two groups of four; group g owns buffer g and the tiles
 // g, g+2, g+4, ... and runs M(i), W(i), U(i) for them, so one group computes while the other
 // waits, and the copies of the tile after next are in flight meanwhile.  A worker's
@@ -55,7 +70,7 @@ constexpr int EP_CONSUMERS = 256;                 // 8 consumer warps
 constexpr int EP_GROUP = EP_CONSUMERS / 2;        // two groups of 4 warps, one per tile buffer
 constexpr int EP_THREADS = EP_CONSUMERS + 32;     // + 1 producer warp
 constexpr int SUB = 8;               // rows per sub-tile
-constexpr int EP_RING = 8;           // partial-margin slots; CTAs are at most 2 tiles apart
+constexpr int EP_RING = 8;           // accumulator slots; a slot is cleared RING/2 tiles before its use
 constexpr int EP_MAX_COLS = 512;     // columns per CTA: 128 groups of 4
 constexpr int EP_BOX_COLS = 256;     // widest TMA box
 constexpr int EP_MAX_M = 256;        // rows per minibatch the fused path takes
@@ -63,6 +78,13 @@ constexpr int EP_MAX_NSUB = EP_MAX_M / SUB;
 constexpr uint64_t DRAIN_LIMIT_NS = 2000000000ull;   // the producer's last wait for its own copies
 constexpr uint64_t COARSE_TIMER_NS = 1024ull;        // limits below this mean "one look, then give up"
 constexpr uint32_t EP_HEADER_WORDS = 64;             // word 0 = abort flag
+constexpr uint32_t EP_ROW_WORDS = 4;                 // 64-bit words per accumulator row (one 32-byte sector)
+constexpr float FX_SCALE = 268435456.0f;             // 2^28: unit of the first word
+constexpr float FX_LIMIT = 131072.0f;                // 2^17: partials below go to the first word
+constexpr float FX_WIDE_SCALE = 64.0f;               // 2^6: unit of the second word
+constexpr float FX_WIDE_LIMIT = 562949953421312.0f;  // 2^49: partials below go to the second word
+constexpr unsigned long long FX_BIAS = 1ull << 45;   // makes every contribution to the first word positive
+constexpr unsigned long long FX_ONE = 1ull << 55;    // one contribution counted
 
 struct EpochArgs {
     const float *y;
@@ -73,13 +95,11 @@ struct EpochArgs {
     uint32_t m_last;        // rows of the last minibatch
     uint32_t nsub_max, nsub_last;
     uint32_t cols;          // columns per CTA, multiple of 4
-    uint32_t gpad;          // CTA count rounded up to a multiple of 32
     float lr;
     float *u;
     uint64_t u_stride;
     uint32_t *header;       // [0] abort flag
-    uint32_t *counters;     // one per tile, zero at launch
-    float *partial;         // [EP_RING][batch][gpad], columns >= gridDim.x stay zero
+    unsigned long long *acc;   // [EP_RING][batch][EP_ROW_WORDS] margin accumulators, zero at launch
     uint32_t *status;
     uint64_t wait_ns;       // limit of every wait on another CTA, warp group or copy
     uint32_t poll_mask;     // the clock is read every (poll_mask + 1) looks at a counter
@@ -158,6 +178,13 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t *p)
 {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ ulonglong2 ld_relaxed_v2(const unsigned long long *p)
+{
+    ulonglong2 v;
+    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "l"(p) : "memory");
     return v;
 }
 
@@ -420,7 +447,14 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
             } else {
                 load_u(T.k, uu);
             }
-            float *__restrict__ pout = a.partial + ((uint64_t)(i % EP_RING) * a.batch) * a.gpad + cta;
+            unsigned long long *const arow = a.acc + (uint64_t)(i % EP_RING) * a.batch * EP_ROW_WORDS;
+            if (cta == i % ncta) {   // this CTA clears the slot that tile i + RING/2 will add into
+                ulonglong2 *z = reinterpret_cast<ulonglong2 *>(
+                    a.acc + (uint64_t)((i + EP_RING / 2) % EP_RING) * a.batch * EP_ROW_WORDS);
+                for (uint32_t j = tg; j < 2u * a.batch; j += EP_GROUP) z[j] = make_ulonglong2(0ull, 0ull);
+                __threadfence();     // cleared for every CTA before this thread goes on
+            }
+            const bool signal = i != 0u || cta != a.drop_cta;
             bool ok = true;
             for (uint32_t s = wg; s < T.nsub; s += EP_GROUP / 32) {   // a warp per sub-tile
                 ok = __all_sync(0xFFFFFFFFu, mbar_wait(&bars[s], parity, &s_flag[0], a.wait_ns)) != 0;
@@ -448,14 +482,25 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
                 }
                 const float tot = reduce8(acc, lane);
                 const uint32_t jj = s * SUB + reduce8_row(lane);
-                if ((lane & 3u) == 0u && jj < T.m) pout[(uint64_t)jj * a.gpad] = tot;
+                if ((lane & 3u) == 0u && jj < T.m && signal) {
+                    unsigned long long *const r = arow + (uint64_t)jj * EP_ROW_WORDS;
+                    if (fabsf(tot) < FX_LIMIT) {
+                        atomicAdd(r, FX_ONE + FX_BIAS + (unsigned long long)__float2ll_rn(tot * FX_SCALE));
+                    } else {
+                        // rare: the wide word or the not-a-number count first, visible before the count
+                        if (fabsf(tot) < FX_WIDE_LIMIT)
+                            atomicAdd(r + 1, (unsigned long long)__float2ll_rn(tot * FX_WIDE_SCALE));
+                        else if (tot != tot)
+                            atomicAdd(r + 2, 1ull);                               // NaN
+                        else
+                            atomicAdd(r + 3, tot > 0.0f ? (1ull << 32) : 1ull);   // +-Inf, or beyond the wide word
+                        __threadfence();
+                        atomicAdd(r, FX_ONE + FX_BIAS);
+                    }
+                }
             }
             if (!ok) s_flag[0] = 1u;
             if (sync_any(1u + g, EP_GROUP, s_flag[0])) break;
-            if (tg == 0) {
-                asm volatile("fence.acq_rel.gpu;" ::: "memory");   // partials before the count
-                if (i != 0u || cta != a.drop_cta) atomicAdd(a.counters + i, 1u);
-            }
         }
 
         // ---- stash: the tile moves from shared to tensor memory and its slots go back to the
@@ -482,10 +527,12 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
         {
             // the labels of the rows this lane will finish, requested before the wait
             const float *__restrict__ yt = a.y + (uint64_t)T.k * a.y_stride + (uint64_t)T.t * a.batch;
-            if (tg == 0) {
+            const unsigned long long *const ain = a.acc + (uint64_t)(i % EP_RING) * a.batch * EP_ROW_WORDS;
+            if (tg == 0) {   // one thread waits for the row that every CTA adds to last
+                const unsigned long long *const last = ain + (uint64_t)(T.m - 1u) * EP_ROW_WORDS;
                 const uint64_t t0 = now_ns();
                 uint32_t n = 0u;
-                while (ld_acquire(a.counters + i) < ncta) {
+                while ((ld_relaxed_v2(last).x >> 55) < ncta) {
                     if ((++n & a.poll_mask) == 0u) {
                         if (s_flag[0] != 0u || ld_acquire(a.header) != 0u || expired(t0, a.wait_ns)) {
                             s_flag[0] = 1u;
@@ -496,42 +543,36 @@ __global__ void __launch_bounds__(EP_THREADS, 1)
                 }
             }
             if (sync_any(1u + g, EP_GROUP, s_flag[0])) break;
-            // a warp sums eight rows at a time: lanes along the CTA index (contiguous in memory)
-            const float *__restrict__ pin = a.partial + ((uint64_t)(i % EP_RING) * a.batch) * a.gpad;
-            // Two passes of eight rows per iteration; all 32 loads of a lane are requested
-            // before the first is used (gpad <= 256).
-            for (uint32_t j0 = wg * SUB; j0 < T.m; j0 += 2u * (EP_GROUP / 32) * SUB) {
-                float4 q0[2][SUB], q1[2][SUB];
-                float yj[2];
-                uint32_t jrow[2];
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint32_t jh = j0 + h * (EP_GROUP / 32) * SUB;
-                    jrow[h] = jh + reduce8_row(lane);
-                    yj[h] = jrow[h] < T.m ? __ldg(yt + jrow[h]) : 0.0f;
-#pragma unroll
-                    for (int r = 0; r < SUB; ++r) {
-                        const float *__restrict__ p = pin + (uint64_t)min(jh + r, T.m - 1u) * a.gpad;
-                        q0[h][r] = q1[h][r] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        if (lane * 4u < a.gpad) q0[h][r] = __ldcg(reinterpret_cast<const float4 *>(p + lane * 4u));
-                        if (128u + lane * 4u < a.gpad)
-                            q1[h][r] = __ldcg(reinterpret_cast<const float4 *>(p + 128u + lane * 4u));
+            // a thread per row: the other rows are complete by now or within a few looks
+            for (uint32_t j = tg; j < T.m; j += EP_GROUP) {
+                const unsigned long long *const r = ain + (uint64_t)j * EP_ROW_WORDS;
+                const float yj = __ldg(yt + j);
+                ulonglong2 v = ld_relaxed_v2(r);
+                if ((v.x >> 55) < ncta) {
+                    const uint64_t t0 = now_ns();
+                    uint32_t n = 0u;
+                    while (((v = ld_relaxed_v2(r)).x >> 55) < ncta) {
+                        if ((++n & a.poll_mask) == 0u &&
+                            (s_flag[0] != 0u || ld_acquire(a.header) != 0u || expired(t0, a.wait_ns))) {
+                            s_flag[0] = 1u;
+                            break;
+                        }
                     }
                 }
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    float v[SUB];
-#pragma unroll
-                    for (int r = 0; r < SUB; ++r)
-                        v[r] = ((q0[h][r].x + q0[h][r].y) + (q0[h][r].z + q0[h][r].w)) +
-                               ((q1[h][r].x + q1[h][r].y) + (q1[h][r].z + q1[h][r].w));
-                    const float margin = reduce8(v, lane);
-                    // -(lr/m) * c_j with c_j = -y_j / (1 + exp(y_j m_j))
-                    if ((lane & 3u) == 0u && jrow[h] < T.m)
-                        coef[jrow[h]] = (a.lr / (float)T.m) * yj[h] / (1.0f + expf(yj[h] * margin));
+                const ulonglong2 special = ld_relaxed_v2(r + 2);   // NaN count | +Inf count << 32 + -Inf count
+                const long long fine = (long long)((v.x & (FX_ONE - 1ull)) - (unsigned long long)ncta * FX_BIAS);
+                float margin = (float)((double)fine * (1.0 / (double)FX_SCALE) +
+                                       (double)(long long)v.y * (1.0 / (double)FX_WIDE_SCALE));
+                if (special.y != 0ull) {
+                    const bool pos = (special.y >> 32) != 0ull, neg = (special.y & 0xFFFFFFFFull) != 0ull;
+                    margin = pos && neg ? __int_as_float(0x7FC00000)
+                                        : __int_as_float(pos ? 0x7F800000 : (int)0xFF800000);
                 }
+                if (special.x != 0ull) margin = __int_as_float(0x7FC00000);
+                // -(lr/m) * c_j with c_j = -y_j / (1 + exp(y_j m_j))
+                coef[j] = (a.lr / (float)T.m) * yj / (1.0f + expf(yj * margin));
             }
-            group_sync();
+            if (sync_any(1u + g, EP_GROUP, s_flag[0])) break;
         }
 
         // ---- U(i): update this CTA's columns of u from the buffer, release the buffer ----
@@ -683,7 +724,7 @@ int qesgd_launch_lr_epoch_fused(const float *X, const float *y, uint64_t n_local
     cols = (cols + 3) / 4 * 4;
     if (cols > (uint64_t)EP_MAX_COLS) return -1;
     const uint32_t ncta = (uint32_t)((d + cols - 1) / cols);
-    if (ncta > 256u) return -1;   // a lane sums at most two groups of four CTAs per row
+    if (ncta > 256u) return -1;   // the accumulator word counts up to 511 contributions
     const int limit = epoch_smem_limit(device);
     if (limit <= 0) return -1;
 
@@ -694,7 +735,6 @@ int qesgd_launch_lr_epoch_fused(const float *X, const float *y, uint64_t n_local
     a.nsub_max = (m_full + SUB - 1) / SUB;
     a.nsub_last = (a.m_last + SUB - 1) / SUB;
     a.cols = (uint32_t)cols;
-    a.gpad = (ncta + 31u) / 32u * 32u;
     a.lr = lr;
     a.u = u; a.u_stride = u_stride;
     a.status = status;
@@ -707,15 +747,11 @@ int qesgd_launch_lr_epoch_fused(const float *X, const float *y, uint64_t n_local
                         (4 * EP_MAX_NSUB) * sizeof(uint64_t) + 64;
     if (smem > (size_t)limit) return -1;
 
-    // workspace: header | one counter per tile | partial margins
-    const uint64_t ntiles = nsteps64 * K;
-    const uint64_t counter_words = (ntiles + 63) / 64 * 64;
-    const uint64_t partial_floats = (uint64_t)EP_RING * m_full * a.gpad;
-    const uint64_t words = EP_HEADER_WORDS + counter_words + partial_floats;
+    // workspace: header | margin accumulators (the workspace is 256-byte aligned)
+    const uint64_t words = EP_HEADER_WORDS + (uint64_t)EP_RING * m_full * EP_ROW_WORDS * 2u;
     if (words > work_floats) return -1;
     a.header = reinterpret_cast<uint32_t *>(work);
-    a.counters = a.header + EP_HEADER_WORDS;
-    a.partial = work + EP_HEADER_WORDS + counter_words;
+    a.acc = reinterpret_cast<unsigned long long *>(work + EP_HEADER_WORDS);
 
     CUtensorMap map_a, map_b;
     const uint32_t cols_a = cols < (uint64_t)EP_BOX_COLS ? (uint32_t)cols : (uint32_t)EP_BOX_COLS;

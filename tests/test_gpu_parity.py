@@ -351,11 +351,61 @@ def test_lr_local_epoch_shapes_match_oracle(K, n_local, d, batch):
         rows = slice(k * n_local, (k + 1) * n_local)
         _lr_close(got[k, :d], ref.lr_local_epoch(X[rows], y[rows], batch, 0.5, u0))
     assert (got[:, d:] == 0).all()
-    # the same call again gives the same bits (fixed summation order, no atomics on data)
+    # the same call again gives the same bits (integer sums between the CTAs, fixed order inside them)
     tu2 = torch.zeros((K, stride), dtype=torch.float32, device="cuda")
     tu2[:, :d] = G.dev(u0)
     c.qesgd_lr_local_epoch_batch(G.dev(X), G.dev(y), n_local, d, K, batch, 0.5, tu2, stride)
     assert torch.equal(tu, tu2)
+
+
+@pytest.mark.parametrize("gain", [2e7, 1e9])
+def test_local_epoch_partial_margins_beyond_the_fine_fixed_point_range(gain):
+    """The CTAs of the persistent kernel add their partial margins as fixed-point integers: units
+    of 2^-28 below 2^17, units of 2^-6 from there on.  With features scaled by 2e7 about half of
+    the partial margins of a row take the coarse word and half the fine one; scaled by 1e9 all
+    take the coarse one (and the second step's reach 1e13).  The oracle knows no such split."""
+    K, n_local, d, batch = 2, 64, 8192, 32
+    X, y, _ = synthetic.logistic_problem(K * n_local, d, seed=31)
+    X = (X * np.float32(gain)).astype(np.float32)
+    u0 = (0.1 * synthetic.normal_f32(d, 1.0, 24)).astype(np.float32)
+    c = G.ctx()
+    tu = torch.zeros((K, d), dtype=torch.float32, device="cuda")
+    tu[:] = G.dev(u0)
+    c.qesgd_lr_local_epoch_batch(G.dev(X), G.dev(y), n_local, d, K, batch, 0.5, tu, d)
+    assert c.qesgd_status() == 0
+    got = tu.cpu().numpy()
+    assert np.isfinite(got).all()
+    for k in range(K):
+        rows = slice(k * n_local, (k + 1) * n_local)
+        _lr_close(got[k], ref.lr_local_epoch(X[rows], y[rows], batch, 0.5, u0))
+
+
+def test_local_epoch_nonfinite_features_spread_as_in_floating_point():
+    """A NaN feature makes its row's margin NaN and with it the worker's whole parameter; an
+    infinite feature makes the margin that infinity, the step coefficient saturates, and only the
+    feature's own column becomes non-finite.  Same pattern as the fp64 oracle; the other worker
+    and the finite entries stay within tolerance."""
+    K, n_local, d, batch = 2, 96, 8192, 32
+    X, y, _ = synthetic.logistic_problem(K * n_local, d, seed=32)
+    u0 = (0.1 * synthetic.normal_f32(d, 1.0, 25)).astype(np.float32)
+    X[40, 1234] = np.nan                     # worker 0, second minibatch
+    X[n_local + 70, 77] = np.inf             # worker 1, last minibatch
+    X[n_local + 80, 4000] = -np.inf
+    c = G.ctx()
+    tu = torch.zeros((K, d), dtype=torch.float32, device="cuda")
+    tu[:] = G.dev(u0)
+    c.qesgd_lr_local_epoch_batch(G.dev(X), G.dev(y), n_local, d, K, batch, 0.5, tu, d)
+    assert c.qesgd_status() == 0
+    got = tu.cpu().numpy()
+    with np.errstate(all="ignore"):
+        want = [ref.lr_local_epoch(X[k * n_local:(k + 1) * n_local], y[k * n_local:(k + 1) * n_local],
+                                   batch, 0.5, u0) for k in range(K)]
+    assert np.isnan(want[0]).all() and np.isnan(got[0]).all()
+    fin = np.isfinite(want[1])
+    assert fin.sum() == d - 2 and not fin[77] and not fin[4000]
+    assert np.array_equal(np.isnan(got[1]), np.isnan(want[1]))
+    assert np.array_equal(got[1][np.isinf(want[1])], want[1][np.isinf(want[1])])
+    _lr_close(got[1][fin], want[1][fin])
 
 
 # ------------------------------ the local-epoch kernel gives up and recovers ---
