@@ -822,8 +822,58 @@ def run_qstep(args, device, world, rank):
                          "peak": peak, "unit": "GB/s", "frac": gbs / peak, "traffic": None,
                          "peak_source": peak_src, "algorithmic_bytes_per_launch": nbytes},
             "status_flags": ctx.qesgd_status(), "clocks": clocks}
+    del u, w, zsum, codes, scales
+    line["inner_step"] = inner_step_leg(ctx, stream, device, args, mode)
     ctx.close()
     return line
+
+
+def inner_step_leg(ctx, stream, device, args, mode):
+    """Algorithm 2's whole inner iteration on logistic regression, m = 64 rows of d = 2^22 columns
+    (a minibatch is 1.07 GB, two of them alternate, so X always comes from HBM): the fused call
+    qesgd_lr_qesgd_step (margin pass + one kernel that updates, quantises and writes back) against
+    qesgd_lr_sgd_step followed by qesgd_requantize (margin pass, update pass, requantise pass)."""
+    import torch
+    from paper_1901_03040_b200 import qesgd, synthetic
+    m, d, B, s, bits, lr = 64, 1 << 22, 512, 127, 8, 0.1
+    X = synthetic.device_normal_f32((2 * m, d), 1.0 / (d ** 0.5), 31, device)
+    y = torch.where(synthetic.device_normal_f32((2 * m,), 1.0, 32, device) >= 0, 1.0, -1.0).float()
+    w = synthetic.device_normal_f32((d,), synthetic.ANCHOR_SIGMA, 33, device)
+    codes, scales = qesgd.alloc_stream_buffers(1, d, B, bits, device)
+    out = {"m": m, "d": d, "bits": bits, "bucket": B}
+    steps = max(args.steps, 10)
+    for name in ("fused", "two_calls"):
+        u = w + synthetic.device_normal_f32((d,), 1e-3, 34, device)
+        zsum = torch.zeros(d, dtype=torch.float32, device=device)
+
+        def call(i):
+            Xb, yb = X[(i % 2) * m:(i % 2 + 1) * m], y[(i % 2) * m:(i % 2 + 1) * m]
+            if name == "fused":
+                ctx.qesgd_lr_qesgd_step(Xb, yb, m, d, lr, u, w, B, s, bits, mode, 7, 0, i, zsum, codes, scales,
+                                        fixed_delta=4e-3 / s)
+            else:
+                ctx.qesgd_lr_sgd_step(Xb, yb, m, d, lr, u)
+                ctx.qesgd_requantize(u, w, d, B, s, bits, mode, 7, 0, i, zsum, codes, scales,
+                                     fixed_delta=4e-3 / s)
+        for i in range(max(args.warmup, 3)):
+            call(i)
+        torch.cuda.synchronize()
+        n0 = ctx.qesgd_launch_count()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            call(i)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        # X twice (margins, update) + u, anchor, running sum read, u and running sum written + code
+        nbytes = 2.0 * m * d * 4 + d * (12.0 + 8.0 + bits / 8.0 + 4.0 / B)
+        out[name] = {"ms_per_step": ms, "launches_per_step": (ctx.qesgd_launch_count() - n0) / steps,
+                     "algorithmic_bytes": nbytes, "hbm_gbs": nbytes / (ms * 1e-3) / 1e9}
+        del u, zsum
+    out["fused_over_two_calls"] = out["fused"]["ms_per_step"] / out["two_calls"]["ms_per_step"]
+    out["status_flags"] = ctx.qesgd_status()
+    return out
 
 
 def run_c1(args, device, world, rank):

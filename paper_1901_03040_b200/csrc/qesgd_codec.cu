@@ -621,14 +621,16 @@ __global__ void __launch_bounds__(WARPS * 32, QESGD_ENCODE_MIN_WARPS / WARPS)
 // added in group order), and its first warp then quantises u^ - w_t, writes u = w_t + Q(z^),
 // the running sum and the stream exactly as qesgd_requantize would.  The updated parameter
 // never travels to global memory before it is quantised.  Buckets of at most 1024 elements,
-// d a multiple of 4, 16-byte aligned X and u.
+// d a multiple of 4, 16-byte aligned X and u.  The register budget is set for three CTAs per SM
+// (the requantising warp needs its 80 registers, the update loop needs the occupancy: with two
+// CTAs per SM the call was 13 % slower than the two separate calls, with three it equals them).
 constexpr int QS_COLS = 256;                   // columns per sub-tile: 64 groups of 4
 constexpr int QS_ROWGROUPS = 4;
 constexpr int QS_THREADS = (QS_COLS / 4) * QS_ROWGROUPS;
 constexpr int QS_TILE = 4 * CHUNK;             // columns per CTA
 
 template <int BITS, int MODE>
-__global__ void __launch_bounds__(QS_THREADS) qesgd_lr_qstep_kernel(const QstepArgs q)
+__global__ void __launch_bounds__(QS_THREADS, 3) qesgd_lr_qstep_kernel(const QstepArgs q)
 {
     __shared__ float s_coef[QESGD_MAX_LR_BATCH];
     __shared__ float4 s_sum[QS_ROWGROUPS][QS_COLS / 4];
@@ -685,6 +687,24 @@ __global__ void __launch_bounds__(QS_THREADS) qesgd_lr_qstep_kernel(const QstepA
     // the first warp requantises the tile: z = u^ - w_t, zeros past d
     const uint32_t lane = threadIdx.x;
     float z[4][8];
+    const bool full = tile0 + QS_TILE <= a.d &&
+                      ((reinterpret_cast<uintptr_t>(a.anchor) | reinterpret_cast<uintptr_t>(a.u_out) |
+                        reinterpret_cast<uintptr_t>(a.zsum)) & 31u) == 0u;
+    if (full) {   // interior tile, aligned vectors: 256-bit loads and stores throughout
+        float w[4][8];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) ld256(a.anchor + tile0 + (uint64_t)c * CHUNK + lane * 8u, w[c]);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const float4 u0 = *reinterpret_cast<const float4 *>(s_u + c * CHUNK + lane * 8u);
+            const float4 u1 = *reinterpret_cast<const float4 *>(s_u + c * CHUNK + lane * 8u + 4u);
+            const float uj[8] = {u0.x, u0.y, u0.z, u0.w, u1.x, u1.y, u1.z, u1.w};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) z[c][j] = __fsub_rn(uj[j], w[c][j]);
+        }
+        encode_warp_tile<BITS, MODE, 4, true, true>(a, z, tile0, 0u, lane, 0u, sh, 0u);
+        return;
+    }
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         const uint64_t e0 = tile0 + (uint64_t)c * CHUNK + lane * 8u;
