@@ -274,9 +274,12 @@ int qesgd_debug_drop_signal(qesgd_ctx *ctx, int64_t cta);
  *     allocation is forbidden, and before starting any stream capture; later calls only
  *     launch two kernels.
  *   - every call shares the one array, which keeps the previous call's contents.
- *     Nothing in it has to start at zero: the first pass overwrites every slot the
- *     second pass reads.  Two calls that overlap on the GPU (different streams, or
- *     different host threads) race on it: serialise them on one stream.
+ *     The first pass overwrites every slot the second pass reads; only the arrival
+ *     counter at the head of the array (by which the last CTA of the first pass knows
+ *     that it is the last) has to be zero between calls: it starts at zero with the
+ *     library image and the kernel that uses it sets it back.  Two calls that overlap
+ *     on the GPU (different streams, or different host threads) race on the array:
+ *     serialise them on one stream.
  */
 int qesgd_lr_sgd_step_noalloc(void *cuda_stream, const float *Xb, const float *yb, uint32_t m,
                               uint64_t d, float lr, float *u);

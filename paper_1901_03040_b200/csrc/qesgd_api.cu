@@ -75,6 +75,8 @@ int qesgd_create(qesgd_ctx **out, int device, void *cuda_stream)
     if (!guard.ok) { delete ctx; return QESGD_ECUDA; }
     cudaError_t e = cudaMalloc((void **)&ctx->d_status, 256);
     if (e == cudaSuccess) e = cudaMalloc((void **)&ctx->d_lr_work, ctx->lr_work_floats * sizeof(float));
+    // the head of the workspace holds arrival counters that the kernels leave at zero
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_lr_work, 0, 256);
     if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
     if (e == cudaSuccess)
         e = cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device);
@@ -239,8 +241,8 @@ int qesgd_lr_qesgd_step(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32
     DeviceGuard guard(ctx->device);
     if (!guard.ok) return cuda_fail(ctx, (int)cudaErrorInvalidDevice);
     QstepArgs q;
-    uint32_t parts = 0;
-    int e = qesgd_launch_lr_margins(Xb, yb, m, d, u, ctx->d_lr_work, ctx->lr_work_floats, ctx->stream, &parts);
+    const float *margins = nullptr;
+    int e = qesgd_launch_lr_margins(Xb, yb, m, d, u, ctx->d_lr_work, ctx->lr_work_floats, ctx->stream, &margins);
     if (e != 0) return cuda_fail(ctx, e);
     ctx->launches += 1;
     EncodeArgs &a = q.e;
@@ -271,8 +273,7 @@ int qesgd_lr_qesgd_step(qesgd_ctx *ctx, const float *Xb, const float *yb, uint32
     q.y = yb;
     q.m = m;
     q.rate = lr / (float)m;
-    q.work = ctx->d_lr_work;
-    q.parts = parts;
+    q.margins = margins;
     switch (bits) {
         case 2: e = qesgd_launch_lr_qstep_2(q, scale_mode, ctx->stream); break;
         case 4: e = qesgd_launch_lr_qstep_4(q, scale_mode, ctx->stream); break;

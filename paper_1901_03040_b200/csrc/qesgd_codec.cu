@@ -638,8 +638,7 @@ __global__ void __launch_bounds__(QS_THREADS, 3) qesgd_lr_qstep_kernel(const Qst
     __shared__ EncodeShared sh;
     const EncodeArgs &a = q.e;
     for (uint32_t j = threadIdx.x; j < q.m; j += blockDim.x) {
-        float margin = 0.0f;
-        for (uint32_t p = 0; p < q.parts; ++p) margin += q.work[(uint64_t)p * q.m + j];
+        const float margin = q.margins[j];
         const float yj = __ldg(q.y + j);
         // -(lr/m) * c_j with c_j = -y_j / (1 + exp(y_j m_j))
         s_coef[j] = q.rate * yj / (1.0f + expf(yj * margin));

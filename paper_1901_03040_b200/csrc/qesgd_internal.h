@@ -62,8 +62,7 @@ struct QstepArgs {
     const float *X, *y;     // the minibatch, m rows of d columns
     uint32_t m;
     float rate;             // lr / m
-    const float *work;      // partial margins of the margin pass: [parts][m]
-    uint32_t parts;
+    const float *margins;   // the m margins, as the margin pass left them
 };
 
 struct DecodeArgs {
@@ -131,7 +130,7 @@ int qesgd_launch_lr_step(const float *Xb, uint64_t x_worker_stride, const float 
 // The margin pass alone (pass 1 of a step) for one worker; *parts_out receives the number of
 // partial margins per row that the pass leaves in `work` ([parts][m]).
 int qesgd_launch_lr_margins(const float *Xb, const float *yb, uint32_t m, uint64_t d, const float *u,
-                            float *work, uint64_t work_floats, cudaStream_t stream, uint32_t *parts_out);
+                            float *work, uint64_t work_floats, cudaStream_t stream, const float **margins_out);
 // Minibatch mean gradient at w into g (same two passes; the second writes instead of updating).
 int qesgd_launch_lr_gradient(const float *Xb, const float *yb, uint32_t m, uint64_t d,
                              const float *w, float *g, float *work, uint64_t work_floats,

@@ -16,7 +16,11 @@
 namespace {
 
 constexpr int SEG = 1024;        // columns per segment in pass 1 (32 lanes x 8 float4)
-constexpr int MAX_PARTS = 64;    // partial-margin slots per worker
+#ifndef QESGD_LR_MAX_PARTS
+#define QESGD_LR_MAX_PARTS 296
+#endif
+constexpr int MAX_PARTS = QESGD_LR_MAX_PARTS;   // CTAs of the margin pass per worker: two per SM of a B200
+constexpr int DONE_WORDS = 64;   // one arrival counter per worker at the head of the workspace
 constexpr int UPD_COLS = 256;      // pass 2: columns per CTA (64 groups of 4)
 constexpr int UPD_ROWGROUPS = 4;   // pass 2: row groups per CTA
 constexpr int UPD_THREADS = (UPD_COLS / 4) * UPD_ROWGROUPS;
@@ -33,7 +37,9 @@ struct LrArgs {
     float *dst;          // accumulate != 0: dst += step (dst == u); else dst = gradient
     uint32_t accumulate;
     uint64_t u_stride;
-    float *work;
+    float *work;         // partial margins [K][P][m]
+    float *margins;      // the margins themselves [K][m], written by the last CTA of each worker
+    uint32_t *done;      // arrival counters [K], zero between launches
     uint32_t parts;      // P
     uint32_t nseg;
 };
@@ -115,6 +121,33 @@ __global__ void __launch_bounds__(256) qesgd_lr_margin_kernel(const LrArgs a)
     __syncthreads();
     float *__restrict__ out = a.work + ((uint64_t)k * a.parts + p) * a.m;
     for (uint32_t j = threadIdx.x; j < a.m; j += blockDim.x) out[j] = s_part[j];
+    // The CTA that arrives last sums the partial margins of its worker, once, in an order that
+    // does not depend on which CTA that is: a row's P partials in four consecutive runs (one
+    // thread each, in index order), the four run sums added in run order.
+    __shared__ uint32_t s_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(a.done + k, 1u) == a.parts - 1u ? 1u : 0u;
+    __syncthreads();
+    if (s_last == 0u) return;
+    __threadfence();
+    const float *__restrict__ w = a.work + (uint64_t)k * a.parts * a.m;
+    const uint32_t run = (a.parts + 3u) / 4u;
+    for (uint32_t j0 = 0; j0 < a.m; j0 += blockDim.x / 4u) {
+        const uint32_t j = j0 + (threadIdx.x >> 2), r = threadIdx.x & 3u;
+        float sum = 0.0f;
+        if (j < a.m) {
+            const uint32_t p0 = r * run, p1 = min(p0 + run, a.parts);
+#pragma unroll 8
+            for (uint32_t q = p0; q < p1; ++q) sum += __ldcg(w + (uint64_t)q * a.m + j);
+        }
+        // lanes 4i .. 4i+3 hold the runs of one row
+        const float s1 = __shfl_down_sync(0xFFFFFFFFu, sum, 1);
+        const float s2 = __shfl_down_sync(0xFFFFFFFFu, sum, 2);
+        const float s3 = __shfl_down_sync(0xFFFFFFFFu, sum, 3);
+        if (r == 0u && j < a.m) a.margins[(uint64_t)k * a.m + j] = ((sum + s1) + s2) + s3;
+    }
+    if (threadIdx.x == 0) a.done[k] = 0u;   // ready for the next launch
 }
 
 // Pass 2.  A CTA updates UPD_COLS consecutive columns: 64 column groups of 4 columns
@@ -129,10 +162,9 @@ __global__ void __launch_bounds__(UPD_THREADS) qesgd_lr_update_kernel(const LrAr
     const float *__restrict__ X = a.X + (uint64_t)k * a.x_stride;
     const float *__restrict__ y = a.y + (uint64_t)k * a.y_stride;
     float *__restrict__ u = a.dst + (uint64_t)k * a.u_stride;
-    const float *__restrict__ work = a.work + (uint64_t)k * a.parts * a.m;
+    const float *__restrict__ margins = a.margins + (uint64_t)k * a.m;
     for (uint32_t j = threadIdx.x; j < a.m; j += blockDim.x) {
-        float margin = 0.0f;
-        for (uint32_t p = 0; p < a.parts; ++p) margin += work[(uint64_t)p * a.m + j];
+        const float margin = margins[j];
         const float yj = __ldg(y + j);
         // -(lr/m) * c_j with c_j = -y_j / (1 + exp(y_j m_j))
         s_coef[j] = a.rate * yj / (1.0f + expf(yj * margin));
@@ -192,6 +224,22 @@ __global__ void __launch_bounds__(UPD_THREADS) qesgd_lr_update_kernel(const LrAr
 
 namespace {
 
+// Workspace: arrival counters | margins [K][m] | partial margins [K][P][m].  P = as many CTAs
+// per worker as the workspace, the segment count and MAX_PARTS allow; 0 if nothing fits.
+uint64_t lay_out_work(LrArgs &a, float *work, uint64_t work_floats, uint32_t K, uint32_t m, uint64_t nseg)
+{
+    const uint64_t head = (uint64_t)DONE_WORDS + (uint64_t)K * m;
+    if (K > (uint32_t)DONE_WORDS || work_floats <= head) return 0;
+    uint64_t parts = (work_floats - head) / ((uint64_t)K * m);
+    if (parts > (uint64_t)MAX_PARTS) parts = MAX_PARTS;
+    if (parts > nseg) parts = nseg;
+    a.done = reinterpret_cast<uint32_t *>(work);
+    a.margins = work + DONE_WORDS;
+    a.work = work + head;
+    a.parts = (uint32_t)parts;
+    return parts;
+}
+
 // Both passes for K workers.  rate multiplies y_j / (1 + exp(y_j m_j)): lr/m for the SGD
 // step (dst = u, accumulated), -1/m for the mean gradient (dst = g, overwritten).
 int launch_lr_passes(const float *Xb, uint64_t x_worker_stride, const float *yb,
@@ -206,13 +254,9 @@ int launch_lr_passes(const float *Xb, uint64_t x_worker_stride, const float *yb,
     a.m = m; a.d = d;
     a.rate = rate;
     a.u = u; a.dst = dst; a.accumulate = accumulate ? 1u : 0u; a.u_stride = u_stride;
-    a.work = work;
     const uint64_t nseg = (d + SEG - 1) / SEG;
-    uint64_t parts = work_floats / ((uint64_t)K * m);
-    if (parts > (uint64_t)MAX_PARTS) parts = MAX_PARTS;
-    if (parts > nseg) parts = nseg;
+    const uint64_t parts = lay_out_work(a, work, work_floats, K, m, nseg);
     if (parts == 0 || nseg > 0xFFFFFFFFull) return (int)cudaErrorInvalidValue;
-    a.parts = (uint32_t)parts;
     a.nseg = (uint32_t)nseg;
     const bool vec = (d % 4 == 0) && (x_worker_stride % 4 == 0) && (u_stride % 4 == 0) &&
                      (((uintptr_t)Xb | (uintptr_t)u | (uintptr_t)dst) % 16 == 0);
@@ -235,7 +279,7 @@ int launch_lr_passes(const float *Xb, uint64_t x_worker_stride, const float *yb,
 }  // namespace
 
 int qesgd_launch_lr_margins(const float *Xb, const float *yb, uint32_t m, uint64_t d, const float *u,
-                            float *work, uint64_t work_floats, cudaStream_t stream, uint32_t *parts_out)
+                            float *work, uint64_t work_floats, cudaStream_t stream, const float **margins_out)
 {
     LrArgs a;
     a.X = Xb; a.x_stride = 0;
@@ -243,19 +287,15 @@ int qesgd_launch_lr_margins(const float *Xb, const float *yb, uint32_t m, uint64
     a.m = m; a.d = d;
     a.rate = 0.0f;
     a.u = u; a.dst = nullptr; a.accumulate = 0u; a.u_stride = 0;
-    a.work = work;
     const uint64_t nseg = (d + SEG - 1) / SEG;
-    uint64_t parts = work_floats / (uint64_t)m;
-    if (parts > (uint64_t)MAX_PARTS) parts = MAX_PARTS;
-    if (parts > nseg) parts = nseg;
+    const uint64_t parts = lay_out_work(a, work, work_floats, 1u, m, nseg);
     if (parts == 0 || nseg > 0xFFFFFFFFull) return (int)cudaErrorInvalidValue;
-    a.parts = (uint32_t)parts;
     a.nseg = (uint32_t)nseg;
     const bool vec = (d % 4 == 0) && (((uintptr_t)Xb | (uintptr_t)u) % 16 == 0);
     dim3 g1((unsigned)parts, 1), b1(256);
     if (vec) qesgd_lr_margin_kernel<true><<<g1, b1, 0, stream>>>(a);
     else qesgd_lr_margin_kernel<false><<<g1, b1, 0, stream>>>(a);
-    *parts_out = a.parts;
+    *margins_out = a.margins;
     return (int)cudaGetLastError();
 }
 
@@ -283,7 +323,7 @@ int qesgd_launch_lr_gradient(const float *Xb, const float *yb, uint32_t m, uint6
 // ---------------------------------------------------------------------------
 namespace {
 
-constexpr uint32_t NOALLOC_FLOATS = MAX_PARTS * QESGD_NOALLOC_MAX_LR_BATCH;   // 64 KB
+constexpr uint32_t NOALLOC_FLOATS = 64 * QESGD_NOALLOC_MAX_LR_BATCH;   // 64 KB: counters, margins, up to 62 parts of 256 rows
 static __device__ __align__(256) float g_noalloc_lr_scratch[NOALLOC_FLOATS];
 
 constexpr int MAX_DEVICES = 64;

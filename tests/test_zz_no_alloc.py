@@ -29,7 +29,8 @@ def test_noalloc_step_matches_the_oracle_and_the_context_entry_point_twice_in_a_
     """Two calls in a row, the second continuing from the first one's result.  Each result is
     compared with the fp64 CPU oracle's step from the same starting point (the tolerance of
     the logistic step, 1e-5) and then with what the context entry point gives.  The last shape
-    (256 rows, 64 column segments) uses every float of the fixed array."""
+    (256 rows, 64 column segments) uses as many partial-margin slots as the fixed array holds
+    (62 of 256 rows beside its counters and margins)."""
     from oracle import qesgd_ref as ref
     torch.cuda.set_device(0)
     X, y, _ = synthetic.logistic_problem(2 * m, d, seed=m + d)
