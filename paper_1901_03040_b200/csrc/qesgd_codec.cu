@@ -31,6 +31,9 @@ constexpr int CHUNK = 256;  // elements covered by one warp-wide 256-bit load
 #ifndef QESGD_DAA_WORDS_WIDE
 #define QESGD_DAA_WORDS_WIDE 2
 #endif
+#ifndef QESGD_DECODE_OCTETS
+#define QESGD_DECODE_OCTETS 4   // octets per thread of the plain decode kernel
+#endif
 #ifndef QESGD_DAA_MIN_CTAS
 #define QESGD_DAA_MIN_CTAS 24   // resident CTAs per SM its register budget is set for
 #endif
@@ -749,39 +752,56 @@ __device__ __forceinline__ void load_codes(const uint8_t *__restrict__ codes, ui
     }
 }
 
+// A thread decodes QESGD_DECODE_OCTETS octets that lie a whole grid apart (so every load and
+// store instruction of a warp stays contiguous); all its code and scale loads are requested
+// before the first is used.  Measured against one octet per thread: 5-14 % faster (four
+// octets; eight are slower again).
 template <int BITS, bool VEC>
 __global__ void __launch_bounds__(256) qesgd_decode_kernel(const DecodeArgs a)
 {
-    const uint64_t eb = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) * 8u;
-    if (eb >= a.d) return;
+    constexpr int OPT = QESGD_DECODE_OCTETS;
+    const uint64_t nthreads = (uint64_t)gridDim.x * blockDim.x;
+    const uint64_t t0 = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const uint8_t *__restrict__ codes = reinterpret_cast<const uint8_t *>(a.codes);
-    uint32_t w[2] = {0u, 0u};
-    float sc = 0.0f;
-    if (QESGD_IN_RANGE(a.status, eb + 8 <= (a.nb << a.log2_bucket))) {
-        load_codes<BITS>(codes, eb, w);
-        sc = __ldg(a.scales + (eb >> a.log2_bucket));
+    uint32_t w[OPT][2];
+    float sc[OPT];
+    uint64_t ebs[OPT];
+#pragma unroll
+    for (int i = 0; i < OPT; ++i) {
+        ebs[i] = (t0 + (uint64_t)i * nthreads) * 8u;
+        w[i][0] = w[i][1] = 0u;
+        sc[i] = 0.0f;
+        if (ebs[i] < a.d && QESGD_IN_RANGE(a.status, ebs[i] + 8 <= (a.nb << a.log2_bucket))) {
+            load_codes<BITS>(codes, ebs[i], w[i]);
+            sc[i] = __ldg(a.scales + (ebs[i] >> a.log2_bucket));
+        }
     }
-    const float step = __fdiv_rn(sc, (float)a.s);
-    float v[8];
-    constexpr int PER_WORD = 32 / BITS;
-    if (BITS == 2) {
-        // A two-bit code moved to bits 31 and 30 IS the float +-2.0 (level 1) or +-0.0 (level 0);
-        // times step/2 (exact: s = 1, so step is the scale, far above the subnormal range or 0)
-        // that is +-step or +-0 bit for bit, the value fl32(level * step) with the code's sign.
-        const float hs = __fmul_rn(step, 0.5f);
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            v[j] = __fmul_rn(__uint_as_float((w[0] << (30 - 2 * j)) & 0xC0000000u), hs);
-    } else {
+    for (int i = 0; i < OPT; ++i) {
+        const uint64_t eb = ebs[i];
+        if (eb >= a.d) continue;
+        const float step = __fdiv_rn(sc[i], (float)a.s);
+        float v[8];
+        constexpr int PER_WORD = 32 / BITS;
+        if (BITS == 2) {
+            // A two-bit code moved to bits 31 and 30 IS the float +-2.0 (level 1) or +-0.0 (level 0);
+            // times step/2 (exact: s = 1, so step is the scale, far above the subnormal range or 0)
+            // that is +-step or +-0 bit for bit, the value fl32(level * step) with the code's sign.
+            const float hs = __fmul_rn(step, 0.5f);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) v[j] = code_value<BITS>(w[j / PER_WORD], j % PER_WORD, step);
-    }
-    if (VEC && eb + 8 <= a.d) {
-        st256(a.param + eb, v);
-    } else {
+            for (int j = 0; j < 8; ++j)
+                v[j] = __fmul_rn(__uint_as_float((w[i][0] << (30 - 2 * j)) & 0xC0000000u), hs);
+        } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j)
-            if (eb + j < a.d) a.param[eb + j] = v[j];
+            for (int j = 0; j < 8; ++j) v[j] = code_value<BITS>(w[i][j / PER_WORD], j % PER_WORD, step);
+        }
+        if (VEC && eb + 8 <= a.d) {
+            st256(a.param + eb, v);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (eb + j < a.d) a.param[eb + j] = v[j];
+        }
     }
 }
 
@@ -1135,7 +1155,7 @@ int QESGD_CAT(qesgd_launch_lr_qstep_, QESGD_BITS)(const QstepArgs &a, uint32_t s
 int QESGD_CAT(qesgd_launch_decode_, QESGD_BITS)(const DecodeArgs &a, bool vec, cudaStream_t stream)
 {
     const uint64_t octets = (a.d + 7) / 8;
-    const uint64_t blocks = (octets + 255) / 256;
+    const uint64_t blocks = (octets + 256 * QESGD_DECODE_OCTETS - 1) / (256 * QESGD_DECODE_OCTETS);
     if (blocks == 0 || blocks > 0x7FFFFFFFull) return (int)cudaErrorInvalidValue;
     dim3 grid((unsigned)blocks), block(256);
     if (vec) qesgd_decode_kernel<QESGD_BITS, true><<<grid, block, 0, stream>>>(a);
