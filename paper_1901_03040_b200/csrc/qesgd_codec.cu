@@ -873,7 +873,7 @@ __device__ __forceinline__ void accumulate_octet(const uint32_t (&cw)[2], int o,
 // completely (no loop counter, no predicates on the worker index).  Measured: 14 % faster for
 // 8-bit, 4 % for 4-bit and 4 % for 2-bit codes at K = 8, but slower for 2-bit codes at K = 4
 // (1 %) and at K = 16 (3-9 %: 16 workers x 32 codes per lane no longer fit the instruction
-// cache); the launcher picks accordingly.
+// cache), where unrolling half the loop gives 2-3 %; the launcher picks accordingly.
 // Register budget: 24 resident CTAs per SM, 28 for 4-bit codes (measured 4-5 % faster there,
 // slower for the other widths).
 template <int BITS, bool VEC, int W, int KS = 0>
@@ -956,7 +956,10 @@ __global__ void __launch_bounds__(QESGD_DAA_THREADS, BITS == 4 ? QESGD_DAA_MIN_C
     fetch(0u, cw);
     float sc_next = fetch_scale(0u);
     float st = 0.0f;
-#pragma unroll
+    // 2-bit codes of 16 workers: two batches per loop iteration (the whole loop would not fit
+    // the instruction cache); every other compile-time worker count: the whole loop
+    constexpr int OUTER_UNROLL = KS == 0 ? 1 : ((BITS == 2 && KS > 8) ? 2 : 64);
+#pragma unroll OUTER_UNROLL
     for (uint32_t kb = 0; kb < (KS ? (uint32_t)KS : a.K); kb += BATCH) {
         fetch(kb + BATCH, nx);
 #pragma unroll
@@ -1177,8 +1180,8 @@ int QESGD_CAT(qesgd_launch_decode_average_apply_, QESGD_BITS)(const DecodeArgs &
         qesgd_decode_average_apply_kernel<QESGD_BITS, true, W, 8><<<grid, block, 0, stream>>>(a);
     else if (vec && QESGD_BITS != 2 && a.K == 4)
         qesgd_decode_average_apply_kernel<QESGD_BITS, true, W, (QESGD_BITS != 2 ? 4 : 0)><<<grid, block, 0, stream>>>(a);
-    else if (vec && QESGD_BITS == 8 && a.K == 16)
-        qesgd_decode_average_apply_kernel<QESGD_BITS, true, W, (QESGD_BITS == 8 ? 16 : 0)><<<grid, block, 0, stream>>>(a);
+    else if (vec && QESGD_BITS != 4 && a.K == 16)
+        qesgd_decode_average_apply_kernel<QESGD_BITS, true, W, (QESGD_BITS != 4 ? 16 : 0)><<<grid, block, 0, stream>>>(a);
     else if (vec) qesgd_decode_average_apply_kernel<QESGD_BITS, true, W><<<grid, block, 0, stream>>>(a);
     else qesgd_decode_average_apply_kernel<QESGD_BITS, false, W><<<grid, block, 0, stream>>>(a);
     return (int)cudaGetLastError();
