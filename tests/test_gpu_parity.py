@@ -298,7 +298,9 @@ def _lr_close(got, want):
 
 
 @pytest.mark.parametrize("m,d", [(64, 4096), (64, 65536), (7, 1000), (1, 5), (200, 3001),
-                                 (1024, 2048)])
+                                 (1024, 2048),
+                                 (16, 524288),     # 512 column segments: every CTA slot of the margin pass in use
+                                 (3, 303108)])     # 297 segments, the last one ragged: one CTA takes two
 def test_lr_step_matches_oracle(m, d):
     X, y, _ = synthetic.logistic_problem(m, d, seed=m + d)
     u = (0.3 * synthetic.normal_f32(d, 1.0, 5)).astype(np.float32)
@@ -552,6 +554,7 @@ def test_qesgd_inner_loop_on_the_gpu_follows_the_oracle():
     (64, 65536, 512, 8, 127, ref.SCALE_NORM, True),    # the benchmark's logistic shape
     (33, 4100, 64, 4, 7, ref.SCALE_MAX, True),         # ragged last tile, odd row count
     (256, 8192, 1024, 2, 1, ref.SCALE_FIXED, True),    # widest bucket the fused kernel takes
+    (16, 524288, 256, 4, 7, ref.SCALE_NORM, True),     # 512 column segments: 296 CTAs in the margin pass
     (64, 8192, 4096, 8, 100, ref.SCALE_NORM, False),   # bucket above 1024: the two calls
     (20, 1002, 128, 4, 7, ref.SCALE_NORM, False),      # d not a multiple of 4: the two calls
 ])

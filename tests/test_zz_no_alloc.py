@@ -24,7 +24,7 @@ def _step_noalloc(X, y, m, d, lr, u):
     assert rc == qesgd.OK, qesgd.lib.qesgd_strerror(rc)
 
 
-@pytest.mark.parametrize("m,d", [(64, 65536), (100, 3001), (256, 4096), (256, 65536)])
+@pytest.mark.parametrize("m,d", [(64, 65536), (100, 3001), (256, 4096), (256, 65536), (16, 524288)])
 def test_noalloc_step_matches_the_oracle_and_the_context_entry_point_twice_in_a_row(m, d):
     """Two calls in a row, the second continuing from the first one's result.  Each result is
     compared with the fp64 CPU oracle's step from the same starting point (the tolerance of
