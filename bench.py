@@ -891,6 +891,21 @@ def inner_step_leg(ctx, stream, device, args, mode):
     return out
 
 
+def c1_kernel_records(times, n, d, K, B, bits):
+    """Mean time of each of the three launches of a C1 round with its algorithmic bytes: every row
+    of X once for the local epoch; locals, anchor and streams for the codec calls."""
+    per = bits / 8.0 + 4.0 / B
+    nbytes = {"local_epoch": float(n) * d * 4, "encode": d * (K * (4 + per) + 4), "apply": d * (K * per + 8)}
+    peak = peaks()[0]
+    out = {}
+    for k, v in times.items():
+        ms = statistics.mean(v)
+        gbs = nbytes[k] / (ms * 1e-3) / 1e9
+        out[k] = {"avg_ms": ms, "min_ms": min(v), "algorithmic_bytes": nbytes[k], "hbm_gbs": gbs,
+                  "frac_of_peak": gbs / peak, "frac_of_8000": gbs / 8000.0}
+    return out
+
+
 def run_c1(args, device, world, rank):
     """End-to-end QESGD round on logistic regression: K=4 workers run one local epoch of
     minibatch-64 SGD from the anchor, encode (8-bit, bucket 512), server applies."""
@@ -947,7 +962,7 @@ def run_c1(args, device, world, rank):
             "config": {"workload": "C1 end-to-end: logistic regression n=8192, d=65536, K=4 workers, "
                                    "one local epoch of minibatch-64 SGD (lr 0.1), 8-bit codes, bucket 512"},
             "gpu_launches": int(ctx.qesgd_launch_count() - launches0),
-            "kernels": {k: {"avg_ms": statistics.mean(v)} for k, v in times.items()},
+            "kernels": c1_kernel_records(times, n, d, K, B, bits),
             "roofline": {"bound": "hbm", "kernel": "qesgd_lr_epoch_kernel (local epoch of all workers)",
                          "achieved": n * d * 4 / (statistics.mean(times["local_epoch"]) * 1e-3) / 1e9,
                          "peak": peaks()[0], "unit": "GB/s",
